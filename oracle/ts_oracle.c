@@ -1,0 +1,225 @@
+/*
+ * CPU oracle for the decode-step hot path -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * Plain, slow, fp64 definitions of what the CUDA library must compute.  Nothing
+ * here is shared with the CUDA path (no common headers, helpers or tables), and
+ * nothing in the product may call into this file: only the tests, the smoke
+ * check and the benchmark's CPU-baseline leg do.
+ *
+ * What is defined (the paper names the operations but prints no formula for
+ * them -- "decode phase" with an active batch, Section 2.1; verification of
+ * draft tokens by the target model in the lossless formulation, Section 3.4 --
+ * so each function below is the textbook definition written out):
+ *
+ *   ora_paged_attention  masked scaled-dot-product attention of q_len query
+ *                        rows per sequence over that sequence's keys, which
+ *                        live in a paged pool addressed through a block table
+ *                        (Section 2.1 decode step; Section 3.4 verify step with
+ *                        q_len = 1 + gamma and a causal mask inside the draft
+ *                        block).  Two passes over a stored score array; no
+ *                        chunking, no running rescale.
+ *   ora_lse_merge        combination of attention results computed over
+ *                        disjoint key subsets, through their log-sum-exp.
+ *   ora_accept_greedy    temperature-0 case of lossless draft verification
+ *                        (Section 3.4): per-row lowest-index argmax over the
+ *                        vocabulary, then the longest draft prefix that agrees
+ *                        with it, plus one token from the target.
+ *
+ * All bf16 inputs are uint16 bit patterns, decoded exactly to double.
+ * Pins for every function live in tests/test_oracle_*.py (brute force on
+ * unpaged tensors written independently in NumPy, closed forms, invariants).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Address of the D-vector of key/value token j of sequence s, kv head g. */
+static const uint16_t *kv_row(const uint16_t *pool, const int32_t *block_table, int64_t max_pages,
+                              int s, int64_t j, int g, int P, int64_t page_stride,
+                              int64_t token_stride, int64_t head_stride)
+{
+    int64_t logical = j / P;
+    int64_t page = block_table[(int64_t)s * max_pages + logical];
+    return pool + page * page_stride + (j % P) * token_stride + (int64_t)g * head_stride;
+}
+
+/*
+ * out : double [B, q_len, Hq, D]      lse : double [B, q_len, Hq] (may be NULL)
+ * key_begin / key_end : optional int32 [B]; when given, only keys j with
+ *   key_begin[s] <= j < key_end[s] take part (used to build split partials).
+ * Query row t of sequence s sits at absolute position n_s - q_len + t and sees
+ * keys 0..that position.  An empty key set yields O = 0 and LSE = -inf.
+ * Returns 0, or -1 on allocation failure / bad arguments.
+ */
+int ora_paged_attention(const uint16_t *q, const uint16_t *k_pool, const uint16_t *v_pool,
+                        const int32_t *block_table, const int32_t *kv_lens,
+                        const int32_t *key_begin, const int32_t *key_end,
+                        int B, int q_len, int Hq, int Hkv, int D, int P, int max_pages,
+                        int64_t page_stride, int64_t token_stride, int64_t head_stride,
+                        double scale, double *out, double *lse, int nthreads)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0 || D <= 0 || P <= 0 || q_len <= 0) return -1;
+    const int G = Hq / Hkv;
+    int failed = 0;
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+#else
+    (void)nthreads;
+#endif
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int s = 0; s < B; ++s) {
+        for (int h = 0; h < Hq; ++h) {
+            const int g = h / G;
+            const int64_t n = kv_lens[s];
+            double *x = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+            if (!x) {
+#pragma omp atomic write
+                failed = 1;
+                continue;
+            }
+            for (int t = 0; t < q_len; ++t) {
+                const uint16_t *qrow = q + (((int64_t)s * q_len + t) * Hq + h) * D;
+                double *orow = out + (((int64_t)s * q_len + t) * Hq + h) * D;
+                const int64_t pos = n - q_len + t;          /* last visible key */
+                int64_t j0 = 0, j1 = pos + 1;               /* visible keys: [j0, j1) */
+                if (key_begin && key_begin[s] > j0) j0 = key_begin[s];
+                if (key_end && key_end[s] < j1) j1 = key_end[s];
+                for (int d = 0; d < D; ++d) orow[d] = 0.0;
+                if (j1 <= j0) {
+                    if (lse) lse[((int64_t)s * q_len + t) * Hq + h] = -INFINITY;
+                    continue;
+                }
+                /* pass 1: scores and their maximum */
+                double m = -INFINITY;
+                for (int64_t j = j0; j < j1; ++j) {
+                    const uint16_t *k = kv_row(k_pool, block_table, max_pages, s, j, g, P,
+                                               page_stride, token_stride, head_stride);
+                    double acc = 0.0;
+                    for (int d = 0; d < D; ++d) acc += bf16_to_double(qrow[d]) * bf16_to_double(k[d]);
+                    x[j] = scale * acc;
+                    if (x[j] > m) m = x[j];
+                }
+                /* pass 2: weights, normaliser, weighted sum of values */
+                double l = 0.0;
+                for (int64_t j = j0; j < j1; ++j) {
+                    const double w = exp(x[j] - m);
+                    l += w;
+                    const uint16_t *v = kv_row(v_pool, block_table, max_pages, s, j, g, P,
+                                               page_stride, token_stride, head_stride);
+                    for (int d = 0; d < D; ++d) orow[d] += w * bf16_to_double(v[d]);
+                }
+                for (int d = 0; d < D; ++d) orow[d] /= l;
+                if (lse) lse[((int64_t)s * q_len + t) * Hq + h] = m + log(l);
+            }
+            free(x);
+        }
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * partial_o   : double [B, max_splits, R, D]   (each already normalised by its own l)
+ * partial_lse : double [B, max_splits, R]      (natural log; -inf marks an empty part)
+ * num_splits  : int32  [B]
+ * out         : double [B, R, D]               R = q_len * Hq rows per sequence
+ * O = sum_i w_i O_i / sum_i w_i with w_i = exp(LSE_i - max_i LSE_i); all parts
+ * empty -> zeros.  out_lse (optional) = max + log(sum w).
+ */
+int ora_lse_merge(const double *partial_o, const double *partial_lse, const int32_t *num_splits,
+                  int B, int max_splits, int R, int D, double *out, double *out_lse)
+{
+    for (int s = 0; s < B; ++s) {
+        const int S = num_splits[s];
+        if (S < 0 || S > max_splits) return -1;
+        for (int r = 0; r < R; ++r) {
+            double *o = out + ((int64_t)s * R + r) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            double M = -INFINITY;
+            for (int i = 0; i < S; ++i) {
+                double v = partial_lse[((int64_t)s * max_splits + i) * R + r];
+                if (v > M) M = v;
+            }
+            if (M == -INFINITY) {
+                if (out_lse) out_lse[(int64_t)s * R + r] = -INFINITY;
+                continue;
+            }
+            double W = 0.0;
+            for (int i = 0; i < S; ++i) {
+                double v = partial_lse[((int64_t)s * max_splits + i) * R + r];
+                if (v == -INFINITY) continue;
+                const double w = exp(v - M);
+                W += w;
+                const double *po = partial_o + (((int64_t)s * max_splits + i) * R + r) * D;
+                for (int d = 0; d < D; ++d) o[d] += w * po[d];
+            }
+            for (int d = 0; d < D; ++d) o[d] /= W;
+            if (out_lse) out_lse[(int64_t)s * R + r] = M + log(W);
+        }
+    }
+    return 0;
+}
+
+/*
+ * logits : bf16 bits, row (b, i) starts at logits + (b*(gamma+1)+i)*row_stride, V entries
+ * draft  : int32 [B, gamma]
+ * target_argmax : int32 [B, gamma+1]   lowest index attaining the row maximum
+ *                 (numeric comparison, so +0 and -0 tie)
+ * accept_len    : int32 [B]            largest a with draft[b,i]==target_argmax[b,i] for all i<a
+ * out_tokens    : int32 [B, gamma+1]   draft[b,:a] ++ target_argmax[b,a], rest -1
+ */
+int ora_accept_greedy(const uint16_t *logits, int64_t row_stride, const int32_t *draft,
+                      int B, int gamma, int V, int32_t *target_argmax, int32_t *accept_len,
+                      int32_t *out_tokens, int nthreads)
+{
+    if (B < 0 || gamma < 0 || V <= 0) return -1;
+    const int R = gamma + 1;
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+#else
+    (void)nthreads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < B * R; ++r) {
+        const uint16_t *row = logits + (int64_t)r * row_stride;
+        int best = 0;
+        double bestv = bf16_to_double(row[0]);
+        for (int v = 1; v < V; ++v) {
+            const double x = bf16_to_double(row[v]);
+            if (x > bestv) { bestv = x; best = v; }
+        }
+        target_argmax[r] = best;
+    }
+    for (int b = 0; b < B; ++b) {
+        int a = 0;
+        while (a < gamma && draft[(int64_t)b * gamma + a] == target_argmax[(int64_t)b * R + a]) ++a;
+        accept_len[b] = a;
+        for (int i = 0; i < R; ++i) {
+            int32_t tok = -1;
+            if (i < a) tok = draft[(int64_t)b * gamma + i];
+            else if (i == a) tok = target_argmax[(int64_t)b * R + a];
+            out_tokens[(int64_t)b * R + i] = tok;
+        }
+    }
+    return 0;
+}
+
+int ora_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
