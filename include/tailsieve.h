@@ -1,0 +1,169 @@
+/*
+ * tailsieve.h -- C ABI of the decode-step kernels that sit under bulk/tail rollout routing.
+ *
+ * The paper routes long ("tail") generations to a low-concurrency pool and the rest to a
+ * high-concurrency ("bulk") pool, and turns on deeper speculative decoding on the tail pool
+ * (Sections 2.1, 3.1, 3.4).  What every replica in either pool executes per step is one batched
+ * decode step over its active requests (Section 2.1: per-request throughput v(b) as a function of
+ * the active batch size b), or, with speculation, one verification of gamma draft tokens by the
+ * target model followed by acceptance (Section 3.4).  This library is the attention and acceptance
+ * part of that step for a ragged batch whose keys and values live in a paged cache.
+ *
+ * General rules (all entry points)
+ *   - Every pointer argument except `const ts_attn_params*` is a DEVICE pointer owned by the
+ *     caller.  The library allocates and frees no device memory, never synchronises the device,
+ *     and only enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - All device pointers must be 16-byte aligned.
+ *   - bf16 tensors are IEEE bfloat16; arithmetic accumulates in fp32.
+ *   - Return value: TS_OK or a negative ts_status.  Argument errors are detected on the host and
+ *     returned before anything is enqueued.  Nothing traps on the device; a device-side wait that
+ *     gives up records TS_ERR_TIMEOUT in the status word at the head of the workspace and the
+ *     kernel returns.
+ *   - One query length per call: every sequence of a batch scores the same number of positions
+ *     (Section 3.4 explains why ragged query lengths are avoided: they break full-batch graph
+ *     replay).
+ *
+ * Tensor conventions
+ *   q        bf16 [num_seqs, q_len, num_q_heads, head_dim], contiguous
+ *   out      bf16 [num_seqs, q_len, num_q_heads, head_dim], contiguous
+ *   k_pool   bf16, element (page p, token j, kv head g, dim d) at
+ *            p*kv_page_stride + j*kv_token_stride + g*kv_head_stride + d   (strides in elements,
+ *            each a multiple of 8 so that every row starts on a 16-byte boundary)
+ *   v_pool   same geometry as k_pool
+ *   block_table int32 [num_seqs, max_pages_per_seq]; entry (s, i) is the physical page holding
+ *            tokens i*page_size .. (i+1)*page_size-1 of sequence s.  Entries at or beyond
+ *            ceil(kv_lens[s] / page_size) are never read.
+ *   kv_lens  int32 [num_seqs]; number of keys of each sequence INCLUDING the q_len positions
+ *            scored by this call (their K/V are already in the cache).  0 is allowed.
+ *   Query head h reads kv head h / (num_q_heads / num_kv_heads).
+ *   Query row t of sequence s stands at position kv_lens[s] - q_len + t and attends to keys
+ *   0 .. that position (causal inside the block of new tokens; all keys when q_len == 1).
+ *   A row with no visible key yields zeros (and -inf as its log-sum-exp).
+ */
+#ifndef TAILSIEVE_H_
+#define TAILSIEVE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum ts_status {
+    TS_OK = 0,
+    TS_ERR_INVALID_ARG = -1, /* null pointer, misaligned pointer, inconsistent sizes            */
+    TS_ERR_UNSUPPORTED = -2, /* head_dim / page_size / group size outside the built set          */
+    TS_ERR_WORKSPACE = -3,   /* workspace smaller than ts_attn_workspace_bytes() and friends     */
+    TS_ERR_CUDA = -4,        /* a CUDA runtime/driver call or a launch failed                    */
+    TS_ERR_TIMEOUT = -5      /* (device status word only) a bounded wait inside a kernel expired */
+} ts_status;
+
+typedef struct ts_attn_params {
+    int32_t num_seqs;          /* B                                                              */
+    int32_t q_len;             /* 1 for decode, 1 + gamma for speculative verification           */
+    int32_t num_q_heads;       /* Hq, a multiple of num_kv_heads                                 */
+    int32_t num_kv_heads;      /* Hkv                                                            */
+    int32_t head_dim;          /* 64 or 128                                                      */
+    int32_t page_size;         /* tokens per page: 16, 32, 64 or 128                             */
+    int32_t num_pages;         /* pages in the pool (extent of the pool's outermost dimension)   */
+    int32_t max_pages_per_seq; /* row stride of block_table                                      */
+    int64_t kv_page_stride;    /* elements                                                       */
+    int64_t kv_token_stride;   /* elements                                                       */
+    int64_t kv_head_stride;    /* elements                                                       */
+    float scale;               /* multiplies q.k in fp32, e.g. 1/sqrt(head_dim)                  */
+} ts_attn_params;
+
+/* Supported shapes: (num_q_heads / num_kv_heads) * q_len <= 96. */
+
+/*
+ * Bytes of scratch that ts_decode_attn / ts_verify_attn need for `p` (depends on the head
+ * geometry and q_len only, not on the sequence lengths).  Host-only; needs no GPU.  Returns 0 for
+ * invalid parameters.
+ */
+size_t ts_attn_workspace_bytes(const ts_attn_params *p);
+
+/* Scratch bytes for ts_decode_attn_splitkv (plan data only; the partials are caller arrays). */
+size_t ts_splitkv_workspace_bytes(const ts_attn_params *p);
+
+/*
+ * Single-token decode attention for one batched decode step (Section 2.1: all active requests
+ * advance by one token per step).  q_len must be 1.
+ *   out = softmax(scale * q K^T) V per (sequence, query head) over that sequence's kv_lens keys.
+ * The key range of long sequences is divided among thread blocks inside the call and recombined;
+ * the result does not depend on how (up to fp32 rounding) and is bit-reproducible run to run.
+ *   workspace: >= ts_attn_workspace_bytes(p) bytes, contents irrelevant on entry, clobbered.
+ *              Its first 4 bytes are a device status word (TS_OK or TS_ERR_TIMEOUT).
+ */
+int ts_decode_attn(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                   const int32_t *block_table, const int32_t *kv_lens, void *out, void *workspace,
+                   size_t workspace_bytes, void *stream);
+
+/*
+ * Attention for the speculative-verification step (Section 3.4: the target model scores the
+ * 1 + gamma positions of each request in one pass).  Same contract as ts_decode_attn with
+ * q_len = 1 + gamma >= 1 and the causal mask inside the block of new tokens described above.
+ */
+int ts_verify_attn(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                   const int32_t *block_table, const int32_t *kv_lens, void *out, void *workspace,
+                   size_t workspace_bytes, void *stream);
+
+/*
+ * Split-KV form of decode attention for a few very long sequences (the tail pool's regime,
+ * Section 3.4: a low-concurrency stream with a long horizon).  Each sequence's keys are cut into
+ * num_splits[s] <= max_splits contiguous ranges, chosen on the device from kv_lens so that the
+ * batch's total work spreads over all SMs; every range is attended to independently.
+ *   partial_o   fp32 [num_seqs, max_splits, q_len, num_q_heads, head_dim]  each range's result,
+ *               normalised by its own softmax denominator
+ *   partial_lse fp32 [num_seqs, max_splits, q_len, num_q_heads]  natural-log sum-exp of the scaled
+ *               scores of the range; -inf when no key of the range is visible to the row
+ *   num_splits  int32 [num_seqs], written with the split counts (>= 1, also for empty sequences,
+ *               whose single slot is written as zeros / -inf)
+ *   workspace   >= ts_splitkv_workspace_bytes(p) bytes, clobbered; first 4 bytes = status word
+ * Only slots i < num_splits[s] are written.  q_len may exceed 1 (same masking as ts_verify_attn).
+ * max_splits in [1, 4096].
+ */
+int ts_decode_attn_splitkv(const ts_attn_params *p, const void *q, const void *k_pool,
+                           const void *v_pool, const int32_t *block_table, const int32_t *kv_lens,
+                           int32_t max_splits, float *partial_o, float *partial_lse,
+                           int32_t *num_splits, void *workspace, size_t workspace_bytes,
+                           void *stream);
+
+/*
+ * Log-sum-exp merge of split results:
+ *   out[s,t,h,:] = sum_i w_i partial_o[s,i,t,h,:] / sum_i w_i,  w_i = exp(lse_i - max_i lse_i),
+ * over i < num_splits[s]; parts with lse = -inf carry zero weight (their partial_o is not read
+ * into the sum); if every part is empty the row is zero.  out is bf16 [num_seqs, q_len,
+ * num_q_heads, head_dim].  Uses num_seqs, q_len, num_q_heads, head_dim of `p` only.
+ */
+int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *partial_o,
+                 const float *partial_lse, const int32_t *num_splits, void *out, void *stream);
+
+/* Scratch bytes for ts_accept_greedy (host-only; 0 for invalid sizes). */
+size_t ts_accept_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab);
+
+/*
+ * Greedy (temperature-0) acceptance of a draft block -- the deterministic case of the lossless
+ * verification rule the paper adopts (Section 3.4).
+ *   logits        bf16; row (b, i), i in [0, gamma], starts at logits + (b*(gamma+1)+i)*row_stride
+ *                 elements and holds `vocab` entries; row_stride >= vocab (rows need not be
+ *                 16-byte aligned; the base pointer must be)
+ *   draft         int32 [num_seqs, gamma]  (may be NULL when gamma == 0)
+ *   target_argmax int32 [num_seqs, gamma+1]  lowest index attaining the row maximum (+0 and -0
+ *                 compare equal; NaN entries never win; a row of -inf or NaN only gives 0)
+ *   accept_len    int32 [num_seqs]  largest a with draft[b,i] == target_argmax[b,i] for all i < a
+ *   out_tokens    int32 [num_seqs, gamma+1] = draft[b,:a] ++ target_argmax[b,a], padded with -1
+ *   workspace     >= ts_accept_workspace_bytes(num_seqs, gamma, vocab) bytes, clobbered
+ * gamma == 0 is plain greedy sampling of one token per sequence.
+ */
+int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draft, int32_t num_seqs,
+                     int32_t gamma, int32_t vocab, int32_t *target_argmax, int32_t *accept_len,
+                     int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Static, human-readable name of a status code. */
+const char *ts_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAILSIEVE_H_ */

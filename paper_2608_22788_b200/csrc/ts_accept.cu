@@ -1,0 +1,186 @@
+// Greedy draft acceptance for sm_100a: a streaming per-row argmax over the vocabulary (HBM-bound,
+// compare-only) followed by the longest-accepted-prefix rule.
+//
+// Kernel 1 cuts every logits row into `chunks` pieces so that even a handful of rows fills the
+// GPU; each CTA reduces its piece to one 64-bit key = (order-preserving image of the bf16 value,
+// ~index), whose maximum is "largest value, lowest index".  Kernel 2 (one CTA) reduces the keys of
+// each row and applies the prefix rule.  No atomics: results are bit-reproducible.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/tailsieve.h"
+
+namespace ts {
+
+constexpr int kArgmaxThreads = 256;
+constexpr int kMaxChunks = 64;
+
+// Order-preserving map of a bf16 bit pattern to an unsigned key: larger value <-> larger key,
+// -0 and +0 share a key, every NaN maps to 0 (below -inf), so NaN never wins.
+__device__ __forceinline__ uint32_t bf16_key(uint32_t u)
+{
+    u &= 0xffffu;
+    if ((u & 0x7fffu) > 0x7f80u) return 0u;          // NaN
+    if (u == 0x8000u) u = 0u;                          // -0 -> +0
+    const uint32_t ord = (u & 0x8000u) ? (~u & 0xffffu) : (u | 0x8000u);
+    return ord + 1u;
+}
+
+__device__ __forceinline__ unsigned long long key_max(unsigned long long a, unsigned long long b)
+{
+    return a > b ? a : b;
+}
+
+__device__ __forceinline__ uint4 ld_stream_16B(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void scan8(const uint4 &v, int idx0, uint32_t &best, int &best_idx)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t k0 = bf16_key(w[i]), k1 = bf16_key(w[i] >> 16);
+        if (k0 > best) { best = k0; best_idx = idx0 + 2 * i; }
+        if (k1 > best) { best = k1; best_idx = idx0 + 2 * i + 1; }
+    }
+}
+
+// grid = (chunks, rows).  keys[row * chunks + chunk] = best key of the chunk.
+__global__ void __launch_bounds__(kArgmaxThreads)
+ts_argmax_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len,
+                       unsigned long long *__restrict__ keys)
+{
+    const int chunk = blockIdx.x, row = blockIdx.y, chunks = gridDim.x;
+    const uint16_t *base = logits + (long long)row * row_stride;
+    const int begin = chunk * chunk_len;
+    int end = begin + chunk_len;
+    if (end > vocab) end = vocab;
+    uint32_t best = 0u;
+    int best_idx = begin < vocab ? begin : 0;
+    // scalar head up to the first 16-byte boundary, 16-byte vectors, scalar tail; every thread
+    // visits its elements in ascending index order, so "strictly greater" keeps the lowest index
+    int head = 0, nvec = 0;
+    if (end > begin) {
+        const long long off = (long long)row * row_stride + begin;
+        head = (int)((8 - (off & 7)) & 7);
+        if (head > end - begin) head = end - begin;
+        nvec = (end - begin - head) / 8;
+    }
+    for (int i = begin + threadIdx.x; i < begin + head; i += kArgmaxThreads) {
+        const uint32_t k = bf16_key(base[i]);
+        if (k > best) { best = k; best_idx = i; }
+    }
+    const int vbeg = begin + head;
+    constexpr int UNROLL = 4;
+    int v = threadIdx.x;
+    for (; v + (UNROLL - 1) * kArgmaxThreads < nvec; v += UNROLL * kArgmaxThreads) {
+        uint4 x[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) x[u] = ld_stream_16B(base + vbeg + (long long)(v + u * kArgmaxThreads) * 8);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) scan8(x[u], vbeg + (v + u * kArgmaxThreads) * 8, best, best_idx);
+    }
+    for (; v < nvec; v += kArgmaxThreads) {
+        const uint4 x = ld_stream_16B(base + vbeg + (long long)v * 8);
+        scan8(x, vbeg + v * 8, best, best_idx);
+    }
+    for (int i = vbeg + nvec * 8 + threadIdx.x; i < end; i += kArgmaxThreads) {
+        const uint32_t k = bf16_key(base[i]);
+        if (k > best) { best = k; best_idx = i; }
+    }
+    unsigned long long key = ((unsigned long long)best << 32) | (unsigned long long)(0xffffffffu - (uint32_t)best_idx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = key_max(key, __shfl_xor_sync(0xffffffffu, key, o));
+    __shared__ unsigned long long wk[kArgmaxThreads / 32];
+    if ((threadIdx.x & 31) == 0) wk[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        key = threadIdx.x < kArgmaxThreads / 32 ? wk[threadIdx.x] : 0ull;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) key = key_max(key, __shfl_xor_sync(0xffffffffu, key, o));
+        if (threadIdx.x == 0) keys[(long long)row * chunks + chunk] = key;
+    }
+}
+
+// One CTA: reduce chunk keys per row, then accept the longest matching draft prefix per sequence.
+__global__ void __launch_bounds__(256)
+ts_accept_finish_kernel(const unsigned long long *__restrict__ keys, int chunks, const int32_t *__restrict__ draft,
+                        int B, int gamma, int32_t *target_argmax, int32_t *accept_len, int32_t *out_tokens)
+{
+    const int R = gamma + 1;
+    for (int r = threadIdx.x; r < B * R; r += blockDim.x) {
+        unsigned long long key = 0ull;
+        for (int c = 0; c < chunks; ++c) key = key_max(key, keys[(long long)r * chunks + c]);
+        target_argmax[r] = (int32_t)(0xffffffffu - (uint32_t)(key & 0xffffffffull));
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        int a = 0;
+        while (a < gamma && draft[(long long)b * gamma + a] == target_argmax[(long long)b * R + a]) ++a;
+        accept_len[b] = a;
+        for (int i = 0; i < R; ++i) {
+            int32_t tok = -1;
+            if (i < a) tok = draft[(long long)b * gamma + i];
+            else if (i == a) tok = target_argmax[(long long)b * R + a];
+            out_tokens[(long long)b * R + i] = tok;
+        }
+    }
+}
+
+static int pick_chunks(long long rows, int vocab)
+{
+    if (rows <= 0) return 1;
+    long long c = (1184 + rows - 1) / rows;       // about 8 CTAs per SM on a 148-SM part
+    const long long by_len = (vocab + 4095) / 4096;   // keep at least ~4096 elements per chunk
+    if (c > by_len) c = by_len;
+    if (c > kMaxChunks) c = kMaxChunks;
+    if (c < 1) c = 1;
+    return (int)c;
+}
+
+}  // namespace ts
+
+extern "C" {
+
+size_t ts_accept_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab)
+{
+    if (num_seqs < 0 || gamma < 0 || vocab < 1) return 0;
+    const long long rows = (long long)num_seqs * (gamma + 1);
+    const size_t bytes = (size_t)rows * ts::kMaxChunks * sizeof(unsigned long long);
+    return bytes < 256 ? 256 : bytes;
+}
+
+int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draft, int32_t num_seqs, int32_t gamma,
+                     int32_t vocab, int32_t *target_argmax, int32_t *accept_len, int32_t *out_tokens, void *workspace,
+                     size_t workspace_bytes, void *stream)
+{
+    if (num_seqs < 0 || gamma < 0 || vocab < 1) return TS_ERR_INVALID_ARG;
+    if (!logits || !target_argmax || !accept_len || !out_tokens || !workspace) return TS_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft) return TS_ERR_INVALID_ARG;
+    if (row_stride < vocab) return TS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(logits) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 15u))
+        return TS_ERR_INVALID_ARG;
+    if (workspace_bytes < ts_accept_workspace_bytes(num_seqs, gamma, vocab)) return TS_ERR_WORKSPACE;
+    const long long rows = (long long)num_seqs * (gamma + 1);
+    if (rows == 0) return TS_OK;
+    if (rows > 65535) return TS_ERR_UNSUPPORTED;
+    const int chunks = ts::pick_chunks(rows, vocab);
+    int chunk_len = (vocab + chunks - 1) / chunks;
+    chunk_len = (chunk_len + 7) / 8 * 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned long long *keys = static_cast<unsigned long long *>(workspace);
+    ts::ts_argmax_chunk_kernel<<<dim3((unsigned)chunks, (unsigned)rows), ts::kArgmaxThreads, 0, s>>>(
+        static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys);
+    if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+    ts::ts_accept_finish_kernel<<<1, 256, 0, s>>>(keys, chunks, draft, num_seqs, gamma, target_argmax, accept_len,
+                                                  out_tokens);
+    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
+}  // extern "C"

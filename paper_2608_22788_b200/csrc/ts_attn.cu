@@ -1,0 +1,1018 @@
+// Paged-KV decode / verify attention for sm_100a.
+//
+// One persistent kernel serves ts_decode_attn, ts_verify_attn and ts_decode_attn_splitkv.
+//
+// Work decomposition.  Every (sequence s, kv head g) pair owns ceil(kv_len_s / 64) KV tiles of 64
+// tokens.  All pairs' tiles are laid end to end in the order (s, g, tile); that line of W tiles is
+// cut into NG equal pieces, one per warp group ("group"; NG = SMs x groups per CTA), so every group
+// streams the same number of bytes whatever the length distribution.  A piece that covers a pair
+// completely produces that pair's final output; a piece that covers only part of a pair writes an
+// fp32 partial (normalised output + log-sum-exp) that a small merge kernel recombines.  In split-KV
+// mode the cuts are moved to the caller-visible per-sequence chunk boundaries instead.
+//
+// Inside a group.  K and V tiles arrive in shared memory through TMA tensor loads (128-byte
+// swizzle) into a ring of stages, each with its own pair of mbarriers; lane 0 of the group's first
+// warp issues them several tiles ahead.  The math runs on warp-level tensor-core MMAs in the
+// "transposed" arrangement: scores S^T[token, row] = K . Q^T with the 64 tokens on the M axis and
+// the G*q_len query rows of the pair on the N axis (8 rows per n-tile), then
+// O^T[dim, row] += V^T . P^T.  That way every byte of K and V is read from shared memory once per
+// warp as an A operand, Q^T lives in registers for the whole segment, and the online-softmax
+// statistics are per-column values a lane already owns.  P is fed to the second MMA as a bf16
+// hi + lo pair so that its rounding stays below the output's own bf16 rounding.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#include "../../include/tailsieve.h"
+#include "ts_common.cuh"
+
+namespace ts {
+
+// ------------------------------------------------------------------------------------------------
+// plan data
+// ------------------------------------------------------------------------------------------------
+struct GroupStart {
+    int32_t s, g, tau, pad;
+};
+
+enum : int { kModeFree = 0, kModeChunks = 1 };
+
+struct AttnArgs {
+    const uint16_t *q;
+    uint16_t *out;
+    const int32_t *block_table;
+    const int32_t *kv_lens;
+    const int32_t *cum_tiles;    // [B+1] exclusive prefix sum of tiles per sequence
+    const GroupStart *gstart;    // [NG+1]
+    const long long *gpos;       // [NG+1] position of each group's first tile on the tile line
+    float *part_o;
+    float *part_lse;
+    const int32_t *num_splits;   // chunk mode: [B]
+    int32_t *status;
+    int B, q_len, Hq, Hkv, G, rows, P, max_pages, max_splits, mode;
+    int ngrp, ns;                // groups per CTA, pipeline stages per group
+    int tok_first;               // 1: token is tensor-map dim 1 and head dim 2; 0: the reverse
+    float scale_log2;            // scale * log2(e)
+    long long wait_cycles;       // bound of every mbarrier wait
+};
+
+__device__ __forceinline__ int div_up(int a, int b) { return (a + b - 1) / b; }
+
+// Largest s in [0, B] with Hkv * cum[s] <= pos.
+__device__ int locate_seq(const int32_t *cum, int B, int Hkv, long long pos)
+{
+    int lo = 0, hi = B;   // invariant: Hkv*cum[lo] <= pos
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((long long)Hkv * cum[mid] <= pos) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// Single-CTA planner: prefix sum of tiles, per-sequence split counts (chunk mode), group starts.
+__global__ void __launch_bounds__(1024, 1)
+ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int mode, int max_splits,
+               int chunks_per_group, int32_t *cum_tiles, GroupStart *gstart, long long *gpos,
+               int32_t *num_splits, int32_t *status, float *part_o, float *part_lse,
+               int rows_all /* q_len*Hq */, int D)
+{
+    __shared__ int warp_sums[32];
+    __shared__ int carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { carry_s = 0; *status = TS_OK; cum_tiles[0] = 0; }
+    __syncthreads();
+    for (int base = 0; base < B; base += 1024) {
+        const int i = base + tid;
+        int v = 0;
+        if (i < B) { const int n = kv_lens[i]; v = n > 0 ? (n + kTile - 1) / kTile : 0; }
+        int x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+        if (lane == 31) warp_sums[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_sums[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += y; }
+            warp_sums[lane] = w;
+        }
+        __syncthreads();
+        const int incl = carry_s + x + (warp > 0 ? warp_sums[warp - 1] : 0);
+        if (i < B) cum_tiles[i + 1] = incl;
+        __syncthreads();
+        if (tid == 1023) carry_s = incl;
+        __syncthreads();
+    }
+    __threadfence_block();
+    __syncthreads();
+    const long long W = (long long)Hkv * cum_tiles[B];
+
+    if (mode == kModeChunks) {
+        long long want = (long long)NG * chunks_per_group;
+        int chunk = (int)((W + want - 1) / want);
+        if (chunk < 1) chunk = 1;
+        for (int s = tid; s < B; s += 1024) {
+            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
+            int S = div_up(tiles, chunk);
+            if (S > max_splits) S = max_splits;
+            if (S < 1) S = 1;
+            if (tiles > 0) { const int ct = div_up(tiles, S); S = div_up(tiles, ct); }
+            num_splits[s] = S;
+        }
+        // empty sequences: their single slot is zeros / -inf
+        for (int s = 0; s < B; ++s) {
+            if (cum_tiles[s + 1] != cum_tiles[s]) continue;
+            float *po = part_o + (size_t)s * max_splits * rows_all * D;
+            float *pl = part_lse + (size_t)s * max_splits * rows_all;
+            for (int i = tid; i < rows_all * D; i += 1024) po[i] = 0.f;
+            for (int i = tid; i < rows_all; i += 1024) pl[i] = -INFINITY;
+        }
+        __threadfence_block();
+        __syncthreads();
+    }
+
+    for (int k = tid; k <= NG; k += 1024) {
+        long long U = (W * k) / NG;
+        int s = locate_seq(cum_tiles, B, Hkv, U);
+        if (mode == kModeChunks && s < B) {
+            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
+            const long long r = U - (long long)Hkv * cum_tiles[s];
+            const int tau = (int)(r % tiles);
+            const int ct = div_up(tiles, num_splits[s]);
+            const int rem = tau % ct;
+            if (rem) {
+                int t2 = tau - rem + ct;
+                if (t2 > tiles) t2 = tiles;
+                U += (t2 - tau);
+                s = locate_seq(cum_tiles, B, Hkv, U);
+            }
+        }
+        GroupStart gs;
+        gs.s = s; gs.g = 0; gs.tau = 0; gs.pad = 0;
+        if (s < B) {
+            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
+            const long long r = U - (long long)Hkv * cum_tiles[s];
+            gs.g = (int)(r / tiles);
+            gs.tau = (int)(r % tiles);
+        }
+        gstart[k] = gs;
+        gpos[k] = U;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// attention kernel
+// ------------------------------------------------------------------------------------------------
+struct Cursor {
+    int s, g, tau, tiles, n;
+};
+
+__device__ __forceinline__ void cur_load(Cursor &c, const AttnArgs &a)
+{
+    if (c.s < a.B) {
+        const int n = a.kv_lens[c.s];
+        c.n = n > 0 ? n : 0;
+        c.tiles = (c.n + kTile - 1) / kTile;
+    } else {
+        c.n = 0;
+        c.tiles = 0;
+    }
+}
+__device__ __forceinline__ void cur_advance(Cursor &c, const AttnArgs &a)
+{
+    if (++c.tau >= c.tiles) {
+        c.tau = 0;
+        if (++c.g >= a.Hkv) {
+            c.g = 0;
+            do { ++c.s; cur_load(c, a); } while (c.s < a.B && c.tiles == 0);
+        }
+    }
+}
+
+template <int D, int NT, int WG>
+__global__ void __launch_bounds__(256, 1)
+ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const AttnArgs a)
+{
+    constexpr int KK = D / 16;            // k-steps of S^T = K Q^T
+    constexpr int MD = D / 16;            // m-tiles (16 dims) of O^T = V^T P^T
+    constexpr int HALVES = D / 64;        // 128-byte swizzle spans per row
+    constexpr int TB = kTile * D * 2;     // bytes of one K (or V) tile
+    constexpr uint32_t FULL = 0xffffffffu;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int ngrp = a.ngrp, ns = a.ns;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp = warp / WG, wig = warp % WG;
+    const int gid = blockIdx.x * ngrp + grp;
+    const uint32_t ring = smem_base + (uint32_t)grp * ns * 2 * TB;
+    const uint32_t bars = smem_base + (uint32_t)ngrp * ns * 2 * TB + (uint32_t)grp * ns * 16;
+    const bool issuer_warp = (wig == 0);
+
+    if (issuer_warp && lane == 0) {
+        for (int st = 0; st < ns; ++st) {
+            mbar_init(bars + st * 16, 1);
+            mbar_init(bars + st * 16 + 8, 1);
+        }
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+    }
+    __syncthreads();
+
+    // ---- this group's piece of the tile line
+    const GroupStart gs = a.gstart[gid];
+    const long long total_ll = a.gpos[gid + 1] - a.gpos[gid];
+    const int total = (int)total_ll;
+    if (total <= 0) return;   // whole group (all its warps) leaves together; no CTA-wide sync follows
+
+    Cursor cc;                 // consume cursor
+    cc.s = gs.s; cc.g = gs.g; cc.tau = gs.tau;
+    cur_load(cc, a);
+    Cursor ic = cc;            // issue cursor
+
+    // ---- page-id prefetch state (issuer warp): 2 x 32 block-table entries in registers
+    int bt_s = -1, bt_base = 0, bt_cur = 0, bt_nxt = 0;
+    bool dead = false;         // set after a wait timed out: later waits are skipped
+
+    const int P = a.P;
+    const int pages_per_tile = P < kTile ? kTile / P : 1;
+    const int tiles_per_page = P > kTile ? P / kTile : 1;
+    const int box_tok = P < kTile ? P : kTile;
+    const uint32_t box_bytes = (uint32_t)box_tok * 128u;
+
+    auto page_id = [&](const Cursor &c, int pg) -> int {
+        const int npages = (c.n + P - 1) / P;
+        const int32_t *row = a.block_table + (size_t)c.s * a.max_pages;
+        if (c.s != bt_s || pg < bt_base || pg >= bt_base + 64) {
+            bt_s = c.s;
+            bt_base = pg & ~31;
+            const int i0 = bt_base + lane, i1 = bt_base + 32 + lane;
+            bt_cur = i0 < npages ? __ldg(row + i0) : 0;
+            bt_nxt = i1 < npages ? __ldg(row + i1) : 0;
+        } else if (pg >= bt_base + 32) {
+            bt_cur = bt_nxt;
+            bt_base += 32;
+            const int i1 = bt_base + 32 + lane;
+            bt_nxt = i1 < npages ? __ldg(row + i1) : 0;
+        }
+        return __shfl_sync(FULL, bt_cur, pg - bt_base);
+    };
+
+    // Issue the TMA loads of the tile under the issue cursor into stage `st` (issuer warp only).
+    auto issue_tile = [&](int st) {
+        const uint32_t kdst = ring + (uint32_t)st * 2 * TB;
+        const uint32_t vdst = kdst + TB;
+        const uint32_t bk = bars + st * 16, bv = bk + 8;
+        int ids[4];
+        int nbox = 1, tok_off = 0;
+        if (P < kTile) {
+            const int first = ic.tau * pages_per_tile;
+            const int npages = (ic.n + P - 1) / P;
+            nbox = npages - first < pages_per_tile ? npages - first : pages_per_tile;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) ids[b] = (b < nbox) ? page_id(ic, first + b) : 0;
+        } else {
+            ids[0] = page_id(ic, ic.tau / tiles_per_page);
+            tok_off = (ic.tau % tiles_per_page) * kTile;
+        }
+        if (lane == 0) {
+            const uint32_t bytes = (uint32_t)nbox * box_bytes * HALVES;
+            mbar_expect_tx(bk, bytes);
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                if (b < nbox) {
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h) {
+                        const int c1 = a.tok_first ? tok_off : ic.g;
+                        const int c2 = a.tok_first ? ic.g : tok_off;
+                        tma_load_4d(kdst + h * (kTile * 128) + b * box_bytes, &tmK, h * 64, c1, c2, ids[b], bk);
+                    }
+                }
+            }
+            mbar_expect_tx(bv, bytes);
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                if (b < nbox) {
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h) {
+                        const int c1 = a.tok_first ? tok_off : ic.g;
+                        const int c2 = a.tok_first ? ic.g : tok_off;
+                        tma_load_4d(vdst + h * (kTile * 128) + b * box_bytes, &tmV, h * 64, c1, c2, ids[b], bv);
+                    }
+                }
+            }
+        }
+    };
+
+    // ---- prologue: fill the ring
+    int issued = 0;
+    if (issuer_warp) {
+        const int pre = total < ns ? total : ns;
+        for (int st = 0; st < pre; ++st) {
+            issue_tile(st);
+            cur_advance(ic, a);
+            ++issued;
+        }
+    }
+
+    // ---- lane-constant pieces of the shared-memory addressing
+    const int l7 = lane & 7;
+    // K (non-transposed ldmatrix): matrices (tok 0-7, chunk c), (tok 8-15, c), (tok 0-7, c+1), (tok 8-15, c+1)
+    const uint32_t k_row_off = (uint32_t)(l7 + ((lane >> 3) & 1) * 8) * 128u;
+    const int k_chunk_l = lane >> 4;
+    // V (transposed ldmatrix): matrices (tok 0-7, chunk c), (tok 0-7, c+1), (tok 8-15, c), (tok 8-15, c+1)
+    const uint32_t v_row_off = (uint32_t)(l7 + (lane >> 4) * 8) * 128u;
+    const int v_chunk_l = (lane >> 3) & 1;
+
+    const int rowbase = wig * 8 * NT;
+    const int qcol = 2 * (lane & 3);         // first of this lane's two columns inside an n-tile
+    const int trow = lane >> 2;              // token (or dim) row inside an 8-row block
+
+    int consumed = 0;                        // tiles consumed so far by this group
+    int remaining = total;
+
+    while (remaining > 0) {
+        // ---------------- segment = run of tiles of one (s, g) pair
+        const int s = cc.s, g = cc.g, tau0 = cc.tau, n = cc.n, tiles = cc.tiles;
+        int seg = tiles - tau0;
+        int chunk_idx = 0;
+        if (a.mode == kModeChunks) {
+            const int ct = div_up(tiles, a.num_splits[s]);
+            chunk_idx = tau0 / ct;
+            const int to_boundary = ct - tau0 % ct;
+            if (to_boundary < seg) seg = to_boundary;
+        }
+        if (remaining < seg) seg = remaining;
+
+        // Q^T fragments of this warp's rows (B operand: k = dim, n = row)
+        uint32_t bq[NT][KK][2];
+        int lim[NT][2];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            const int r = rowbase + 8 * j + trow;
+            const bool valid = r < a.rows;
+            const int t = valid ? r / a.G : 0, hl = valid ? r % a.G : 0;
+            const uint16_t *qp = a.q + (((size_t)s * a.q_len + t) * a.Hq + (size_t)g * a.G + hl) * D + qcol;
+#pragma unroll
+            for (int kk = 0; kk < KK; ++kk) {
+                bq[j][kk][0] = valid ? __ldg(reinterpret_cast<const uint32_t *>(qp + 16 * kk)) : 0u;
+                bq[j][kk][1] = valid ? __ldg(reinterpret_cast<const uint32_t *>(qp + 16 * kk + 8)) : 0u;
+            }
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int rc = rowbase + 8 * j + qcol + e;
+                lim[j][e] = rc < a.rows ? n - a.q_len + rc / a.G : -1;   // last visible token index
+            }
+        }
+
+        float m_run[NT][2], l_run[NT][2];
+        float acc_o[MD][NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) { m_run[j][0] = m_run[j][1] = -INFINITY; l_run[j][0] = l_run[j][1] = 0.f; }
+#pragma unroll
+        for (int md = 0; md < MD; ++md)
+#pragma unroll
+            for (int j = 0; j < NT; ++j) { acc_o[md][j][0] = acc_o[md][j][1] = acc_o[md][j][2] = acc_o[md][j][3] = 0.f; }
+
+        for (int tau = tau0; tau < tau0 + seg; ++tau) {
+            const int st = consumed % ns;
+            const uint32_t parity = (uint32_t)(consumed / ns) & 1u;
+            const uint32_t kbase = ring + (uint32_t)st * 2 * TB;
+            const uint32_t vbase = kbase + TB;
+            const uint32_t bk = bars + st * 16, bv = bk + 8;
+            const int tok0 = tau * kTile;
+
+            // ---------- S^T = K Q^T
+            if (!dead && !mbar_wait_bounded(bk, parity, a.wait_cycles)) { dead = true; atomicExch(a.status, (int)TS_ERR_TIMEOUT); }
+            float sacc[4][NT][4];
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int j = 0; j < NT; ++j) { sacc[mi][j][0] = sacc[mi][j][1] = sacc[mi][j][2] = sacc[mi][j][3] = 0.f; }
+#pragma unroll
+            for (int kk = 0; kk < KK; ++kk) {
+                const int chunk = 2 * kk + k_chunk_l;
+                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (kTile * 128);
+#pragma unroll
+                for (int mi = 0; mi < 4; ++mi) {
+                    uint32_t af[4];
+                    ldsm_x4(af, kbase + mi * 2048 + k_row_off + col);
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) mma_bf16_16816(sacc[mi][j], af, bq[j][kk][0], bq[j][kk][1]);
+                }
+            }
+
+            // ---------- online softmax (per column = query row)
+            const bool need_mask = tok0 + kTile - 1 > n - a.q_len;
+            float mx[NT][2];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) { mx[j][0] = mx[j][1] = -INFINITY; }
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        float x = sacc[mi][j][r] * a.scale_log2;
+                        if (need_mask) {
+                            const int tok = tok0 + 16 * mi + trow + ((r >> 1) << 3);
+                            if (tok > lim[j][r & 1]) x = -INFINITY;
+                        }
+                        sacc[mi][j][r] = x;
+                        mx[j][r & 1] = fmaxf(mx[j][r & 1], x);
+                    }
+            float alpha[NT][2], mref[NT][2];
+            bool changed = false;
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float v = mx[j][e];
+                    v = fmaxf(v, __shfl_xor_sync(FULL, v, 4));
+                    v = fmaxf(v, __shfl_xor_sync(FULL, v, 8));
+                    v = fmaxf(v, __shfl_xor_sync(FULL, v, 16));
+                    const float m_new = fmaxf(m_run[j][e], v);
+                    mref[j][e] = (m_new == -INFINITY) ? 0.f : m_new;
+                    alpha[j][e] = ex2(m_run[j][e] - mref[j][e]);     // m_run = -inf -> 0
+                    changed |= (m_new != m_run[j][e]);
+                    m_run[j][e] = m_new;
+                    l_run[j][e] *= alpha[j][e];
+                }
+            if (__any_sync(FULL, changed)) {
+#pragma unroll
+                for (int md = 0; md < MD; ++md)
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        acc_o[md][j][0] *= alpha[j][0]; acc_o[md][j][1] *= alpha[j][1];
+                        acc_o[md][j][2] *= alpha[j][0]; acc_o[md][j][3] *= alpha[j][1];
+                    }
+            }
+            // P^T fragments (B operand of the second MMA: k = token, n = row), bf16 hi + lo
+            uint32_t bph[4][NT][2], bpl[4][NT][2];
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    float p[4];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        p[r] = ex2(sacc[mi][j][r] - mref[j][r & 1]);
+                        l_run[j][r & 1] += p[r];
+                    }
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const uint32_t hi = pack_bf16x2(p[2 * hh], p[2 * hh + 1]);
+                        const uint32_t lo = pack_bf16x2(p[2 * hh] - bf16lo_to_f32(hi), p[2 * hh + 1] - bf16hi_to_f32(hi));
+                        bph[mi][j][hh] = movmatrix_trans(hi);
+                        bpl[mi][j][hh] = movmatrix_trans(lo);
+                    }
+                }
+
+            // ---------- O^T += V^T P^T
+            if (!dead && !mbar_wait_bounded(bv, parity, a.wait_cycles)) { dead = true; atomicExch(a.status, (int)TS_ERR_TIMEOUT); }
+            const int valid_tok = n - tok0;          // tokens of this tile that exist
+            if (valid_tok < kTile) {
+                // rows past the sequence end may hold anything (also NaN): zero them so that 0 * v = 0
+                for (int r = valid_tok + (lane >> 3); r < kTile; r += 4)
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h) {
+                        const uint32_t addr = vbase + h * (kTile * 128) + r * 128 + l7 * 16;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                    }
+                __syncwarp();
+            }
+#pragma unroll
+            for (int md = 0; md < MD; ++md) {
+                const int chunk = 2 * md + v_chunk_l;
+                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (kTile * 128);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t af[4];
+                    ldsm_x4_trans(af, vbase + ks * 2048 + v_row_off + col);
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        mma_bf16_16816(acc_o[md][j], af, bph[ks][j][0], bph[ks][j][1]);
+                        mma_bf16_16816(acc_o[md][j], af, bpl[ks][j][0], bpl[ks][j][1]);
+                    }
+                }
+            }
+
+            // ---------- release the stage and refill it
+            if (valid_tok < kTile) fence_proxy_async_smem();
+            if (WG == 1) __syncwarp(); else named_bar_sync(1 + grp, WG * 32);
+            ++consumed;
+            if (issuer_warp && issued < total) {
+                issue_tile(st);
+                cur_advance(ic, a);
+                ++issued;
+            }
+        }
+
+        // ---------------- epilogue of the segment
+        const bool full_pair = (tau0 == 0 && seg == tiles);
+        const bool write_final = (a.mode == kModeFree) && full_pair;
+        size_t slot = 0;
+        if (a.mode == kModeFree) slot = (size_t)2 * gid + (tau0 > 0 ? 0 : 1);
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                float l = l_run[j][e];
+                l += __shfl_xor_sync(FULL, l, 4);
+                l += __shfl_xor_sync(FULL, l, 8);
+                l += __shfl_xor_sync(FULL, l, 16);
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const int rc = rowbase + 8 * j + qcol + e;
+                if (rc >= a.rows) continue;
+                const int t = rc / a.G, hl = rc % a.G;
+                const size_t row_th = ((size_t)s * a.q_len + t) * a.Hq + (size_t)g * a.G + hl;   // (s, t, h) flat
+                if (write_final) {
+                    uint16_t *op = a.out + row_th * D;
+#pragma unroll
+                    for (int md = 0; md < MD; ++md) {
+                        const float v0 = acc_o[md][j][e] * inv, v1 = acc_o[md][j][2 + e] * inv;
+                        const uint32_t pk = pack_bf16x2(v0, v1);
+                        op[16 * md + trow] = (uint16_t)(pk & 0xffffu);
+                        op[16 * md + trow + 8] = (uint16_t)(pk >> 16);
+                    }
+                } else {
+                    float *po, *pl;
+                    if (a.mode == kModeFree) {
+                        po = a.part_o + (slot * a.rows + rc) * D;
+                        pl = a.part_lse + slot * a.rows + rc;
+                    } else {
+                        const size_t rows_all = (size_t)a.q_len * a.Hq;
+                        const size_t base = ((size_t)s * a.max_splits + chunk_idx) * rows_all + ((size_t)t * a.Hq + (size_t)g * a.G + hl);
+                        po = a.part_o + base * D;
+                        pl = a.part_lse + base;
+                    }
+#pragma unroll
+                    for (int md = 0; md < MD; ++md) {
+                        po[16 * md + trow] = acc_o[md][j][e] * inv;
+                        po[16 * md + trow + 8] = acc_o[md][j][2 + e] * inv;
+                    }
+                    if (trow == 0) *pl = l > 0.f ? (m_run[j][e] + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+
+        remaining -= seg;
+        cc.tau += seg - 1;
+        cur_advance(cc, a);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// merge kernels
+// ------------------------------------------------------------------------------------------------
+// One warp merges one output row: `count` parts, part i at po + i*o_stride / pl + i*l_stride.
+template <int D>
+__device__ __forceinline__ void merge_row(const float *po, size_t o_stride, const float *pl, size_t l_stride,
+                                          int count, uint16_t *out_row, int lane)
+{
+    constexpr int V = D / 32;     // floats per lane
+    float M = -INFINITY;
+    for (int i = 0; i < count; ++i) M = fmaxf(M, pl[(size_t)i * l_stride]);
+    float acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = 0.f;
+    float Wsum = 0.f;
+    if (M != -INFINITY) {
+        for (int i = 0; i < count; ++i) {
+            const float lse = pl[(size_t)i * l_stride];
+            if (lse == -INFINITY) continue;
+            const float w = expf(lse - M);
+            Wsum += w;
+            const float *p = po + (size_t)i * o_stride + lane * V;
+#pragma unroll
+            for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+        }
+    }
+    const float inv = Wsum > 0.f ? 1.f / Wsum : 0.f;
+    uint16_t *o = out_row + lane * V;
+#pragma unroll
+    for (int v = 0; v < V; v += 2) {
+        const uint32_t pk = pack_bf16x2(acc[v] * inv, acc[v + 1] * inv);
+        *reinterpret_cast<uint32_t *>(o + v) = pk;
+    }
+}
+
+// Free mode: one CTA (4 warps) per (s, g) pair; pairs covered by a single group are skipped.
+template <int D>
+__global__ void __launch_bounds__(128)
+ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restrict__ part_o,
+                     const float *__restrict__ part_lse, uint16_t *out, int B, int q_len, int Hq, int Hkv,
+                     int NG)
+{
+    const int pair = blockIdx.x;
+    const int s = pair / Hkv, g = pair % Hkv;
+    const int G = Hq / Hkv, rows = G * q_len;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles = cum_tiles[s + 1] - cum_tiles[s];
+    const long long W = (long long)Hkv * cum_tiles[B];
+    int k_first = 0, k_last = -1;
+    if (tiles > 0) {
+        const long long a0 = (long long)Hkv * cum_tiles[s] + (long long)g * tiles, b0 = a0 + tiles;
+        k_first = (int)(((a0 + 1) * NG - 1) / W);
+        k_last = (int)((b0 * NG - 1) / W);
+        if (k_first == k_last) return;      // written directly by the attention kernel
+    }
+    for (int r = warp; r < rows; r += 4) {
+        const int t = r / G, hl = r % G;
+        uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
+        if (tiles == 0) {
+            merge_row<D>(nullptr, 0, nullptr, 0, 0, orow, lane);
+            continue;
+        }
+        // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
+        // (pair started before them).
+        // Groups whose piece of the tile line is empty (only when W < NG) wrote nothing: skip them.
+        float M = -INFINITY;
+        for (int k = k_first; k <= k_last; ++k) {
+            if ((W * k) / NG == (W * (k + 1)) / NG) continue;
+            const size_t slot = (size_t)2 * k + (k == k_first ? 1 : 0);
+            M = fmaxf(M, part_lse[slot * rows + r]);
+        }
+        constexpr int V = D / 32;
+        float acc[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[v] = 0.f;
+        float Wsum = 0.f;
+        if (M != -INFINITY) {
+            for (int k = k_first; k <= k_last; ++k) {
+                if ((W * k) / NG == (W * (k + 1)) / NG) continue;
+                const size_t slot = (size_t)2 * k + (k == k_first ? 1 : 0);
+                const float lse = part_lse[slot * rows + r];
+                if (lse == -INFINITY) continue;
+                const float w = expf(lse - M);
+                Wsum += w;
+                const float *p = part_o + (slot * rows + r) * D + lane * V;
+#pragma unroll
+                for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+            }
+        }
+        const float inv = Wsum > 0.f ? 1.f / Wsum : 0.f;
+        uint16_t *o = orow + lane * V;
+#pragma unroll
+        for (int v = 0; v < V; v += 2) *reinterpret_cast<uint32_t *>(o + v) = pack_bf16x2(acc[v] * inv, acc[v + 1] * inv);
+    }
+}
+
+// Caller-visible dense layout: one warp per output row (s, t, h).
+template <int D>
+__global__ void __launch_bounds__(128)
+ts_merge_dense_kernel(const float *__restrict__ part_o, const float *__restrict__ part_lse,
+                      const int32_t *__restrict__ num_splits, uint16_t *out, int B, int rows_all, int max_splits)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 4 + warp;
+    if (row >= (long long)B * rows_all) return;
+    const int s = (int)(row / rows_all), r = (int)(row % rows_all);
+    int S = num_splits[s];
+    if (S > max_splits) S = max_splits;
+    if (S < 0) S = 0;
+    const float *po = part_o + ((size_t)s * max_splits * rows_all + r) * D;
+    const float *pl = part_lse + (size_t)s * max_splits * rows_all + r;
+    merge_row<D>(po, (size_t)rows_all * D, pl, (size_t)rows_all, S, out + (size_t)row * D, lane);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+    size_t status, cum_tiles, gstart, gpos, part_lse, part_o, total;
+};
+
+static WorkspaceLayout layout_workspace(const ts_attn_params *p, bool with_partials)
+{
+    WorkspaceLayout w;
+    const size_t rows = (size_t)(p->num_q_heads / p->num_kv_heads) * p->q_len;
+    size_t off = 0;
+    w.status = off; off += 256;
+    w.cum_tiles = off; off = align_up(off + ((size_t)p->num_seqs + 1) * 4, 256);
+    w.gstart = off; off = align_up(off + ((size_t)kMaxGroups + 1) * sizeof(GroupStart), 256);
+    w.gpos = off; off = align_up(off + ((size_t)kMaxGroups + 1) * 8, 256);
+    w.part_lse = off;
+    if (with_partials) off = align_up(off + (size_t)2 * kMaxGroups * rows * 4, 256);
+    w.part_o = off;
+    if (with_partials) off = align_up(off + (size_t)2 * kMaxGroups * rows * p->head_dim * 4, 256);
+    w.total = off;
+    return w;
+}
+
+static int check_params(const ts_attn_params *p)
+{
+    if (!p) return TS_ERR_INVALID_ARG;
+    if (p->num_seqs < 0 || p->q_len < 1 || p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_pages < 1 ||
+        p->max_pages_per_seq < 1)
+        return TS_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads != 0) return TS_ERR_INVALID_ARG;
+    if (p->kv_page_stride <= 0 || p->kv_token_stride <= 0 || p->kv_head_stride <= 0) return TS_ERR_INVALID_ARG;
+    if (p->kv_page_stride % 8 || p->kv_token_stride % 8 || p->kv_head_stride % 8) return TS_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return TS_ERR_UNSUPPORTED;
+    if (p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128) return TS_ERR_UNSUPPORTED;
+    const long long rows = (long long)(p->num_q_heads / p->num_kv_heads) * p->q_len;
+    if (rows > kMaxRows) return TS_ERR_UNSUPPORTED;
+    if (!(p->scale == p->scale) || isinf(p->scale)) return TS_ERR_INVALID_ARG;
+    return TS_OK;
+}
+
+static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_params *p, int *tok_first)
+{
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return TS_ERR_CUDA;
+    // dims: 0 = head_dim, then {token, head} by ascending stride, then page
+    const bool tf = p->kv_token_stride <= p->kv_head_stride;
+    *tok_first = tf ? 1 : 0;
+    cuuint64_t dims[4], strides[3];
+    cuuint32_t box[4], estr[4] = {1, 1, 1, 1};
+    const cuuint32_t box_tok = (cuuint32_t)(p->page_size < kTile ? p->page_size : kTile);
+    dims[0] = (cuuint64_t)p->head_dim;
+    box[0] = 64;
+    if (tf) {
+        dims[1] = (cuuint64_t)p->page_size; strides[0] = (cuuint64_t)p->kv_token_stride * 2; box[1] = box_tok;
+        dims[2] = (cuuint64_t)p->num_kv_heads; strides[1] = (cuuint64_t)p->kv_head_stride * 2; box[2] = 1;
+    } else {
+        dims[1] = (cuuint64_t)p->num_kv_heads; strides[0] = (cuuint64_t)p->kv_head_stride * 2; box[1] = 1;
+        dims[2] = (cuuint64_t)p->page_size; strides[1] = (cuuint64_t)p->kv_token_stride * 2; box[2] = box_tok;
+    }
+    dims[3] = (cuuint64_t)p->num_pages; strides[2] = (cuuint64_t)p->kv_page_stride * 2; box[3] = 1;
+    const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TS_OK : TS_ERR_UNSUPPORTED;
+}
+
+struct DeviceInfo {
+    int sms = 0;
+    int smem_optin = 0;
+    int clock_khz = 0;
+    bool ok = false;
+};
+
+static const DeviceInfo &device_info()
+{
+    static DeviceInfo info[64];
+    static DeviceInfo bad;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return bad;
+    DeviceInfo &d = info[dev];
+    if (!d.ok) {
+        if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return bad;
+        if (cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return bad;
+        if (cudaDeviceGetAttribute(&d.clock_khz, cudaDevAttrClockRate, dev) != cudaSuccess) d.clock_khz = 2000000;
+        d.ok = d.sms > 0;
+    }
+    return d;
+}
+
+static int env_int(const char *name, int dflt)
+{
+    const char *v = getenv(name);
+    if (!v || !*v) return dflt;
+    return atoi(v);
+}
+
+template <int D, int NT, int WG>
+static int launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a, int sms, int smem_optin,
+                       cudaStream_t stream, bool dry, int *ng_out)
+{
+    constexpr int TB = kTile * D * 2;
+    // groups per CTA and stages per group: as much shared memory in flight as fits, at most 256 threads
+    int ngrp = env_int("TS_ATTN_NGRP", WG == 1 ? 3 : (WG == 2 ? 3 : 2));
+    if (ngrp * WG * 32 > 256) ngrp = 256 / (WG * 32);
+    if (ngrp < 1) ngrp = 1;
+    int ns = env_int("TS_ATTN_STAGES", 0);
+    const int budget = smem_optin - 2048;
+    if (ns <= 0) ns = budget / (ngrp * 2 * TB);
+    if (ns > 8) ns = 8;
+    while (ns > 1 && (size_t)ngrp * ns * 2 * TB + 1024 + (size_t)ngrp * ns * 16 > (size_t)budget) --ns;
+    if (ns < 2) { ngrp = 1; ns = 2; }
+    const size_t smem = (size_t)ngrp * ns * 2 * TB + (size_t)ngrp * ns * 16 + 1024;
+    if (smem > (size_t)smem_optin) return TS_ERR_UNSUPPORTED;
+    int grid = sms;
+    const int grid_cap = env_int("TS_ATTN_GRID", 0);      // testing knob: fewer CTAs, longer pieces
+    if (grid_cap > 0 && grid_cap < grid) grid = grid_cap;
+    if ((long long)grid * ngrp > kMaxGroups) grid = kMaxGroups / ngrp;
+    *ng_out = grid * ngrp;
+    a.ngrp = ngrp;
+    a.ns = ns;
+    if (dry) return TS_OK;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(ts_attn_kernel<D, NT, WG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
+            return TS_ERR_CUDA;
+        attr_set = true;
+    }
+    ts_attn_kernel<D, NT, WG><<<grid, ngrp * WG * 32, smem, stream>>>(tk, tv, a);
+    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
+template <int D>
+static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a, int sms, int smem_optin,
+                         cudaStream_t stream, bool dry, int *ng)
+{
+    if (rows <= 8) return launch_attn<D, 1, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    if (rows <= 16) return launch_attn<D, 2, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    if (rows <= 24) return launch_attn<D, 3, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    if (rows <= 48) return launch_attn<D, 3, 2>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    if (rows <= 72) return launch_attn<D, 3, 3>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    if (rows <= 96) return launch_attn<D, 3, 4>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    return TS_ERR_UNSUPPORTED;
+}
+
+// Shared driver of the three attention entry points.
+static int run_attention(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                         const int32_t *block_table, const int32_t *kv_lens, int mode, int max_splits, void *out,
+                         float *part_o, float *part_lse, int32_t *num_splits, void *workspace, size_t workspace_bytes,
+                         void *stream_v)
+{
+    int rc = check_params(p);
+    if (rc != TS_OK) return rc;
+    if (!q || !k_pool || !v_pool || !block_table || !kv_lens || !workspace) return TS_ERR_INVALID_ARG;
+    if (misaligned(q) || misaligned(k_pool) || misaligned(v_pool) || misaligned(block_table) || misaligned(kv_lens) ||
+        misaligned(workspace))
+        return TS_ERR_INVALID_ARG;
+    const bool free_mode = (mode == kModeFree);
+    if (free_mode) {
+        if (!out || misaligned(out)) return TS_ERR_INVALID_ARG;
+    } else {
+        if (!part_o || !part_lse || !num_splits || misaligned(part_o) || misaligned(part_lse) || misaligned(num_splits))
+            return TS_ERR_INVALID_ARG;
+        if (max_splits < 1 || max_splits > 4096) return TS_ERR_INVALID_ARG;
+    }
+    const WorkspaceLayout w = layout_workspace(p, free_mode);
+    if (workspace_bytes < w.total) return TS_ERR_WORKSPACE;
+    if (p->num_seqs == 0) return TS_OK;
+
+    const DeviceInfo &dev = device_info();
+    if (!dev.ok) return TS_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+
+    CUtensorMap tk, tv;
+    int tok_first = 1, tf2 = 1;
+    rc = make_tensor_map(&tk, k_pool, p, &tok_first);
+    if (rc != TS_OK) return rc;
+    rc = make_tensor_map(&tv, v_pool, p, &tf2);
+    if (rc != TS_OK) return rc;
+
+    AttnArgs a;
+    a.q = static_cast<const uint16_t *>(q);
+    a.out = static_cast<uint16_t *>(out);
+    a.block_table = block_table;
+    a.kv_lens = kv_lens;
+    a.cum_tiles = reinterpret_cast<const int32_t *>(ws + w.cum_tiles);
+    a.gstart = reinterpret_cast<const GroupStart *>(ws + w.gstart);
+    a.gpos = reinterpret_cast<const long long *>(ws + w.gpos);
+    a.part_o = free_mode ? reinterpret_cast<float *>(ws + w.part_o) : part_o;
+    a.part_lse = free_mode ? reinterpret_cast<float *>(ws + w.part_lse) : part_lse;
+    a.num_splits = num_splits;
+    a.status = reinterpret_cast<int32_t *>(ws + w.status);
+    a.B = p->num_seqs; a.q_len = p->q_len; a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads;
+    a.G = p->num_q_heads / p->num_kv_heads; a.rows = a.G * p->q_len; a.P = p->page_size;
+    a.max_pages = p->max_pages_per_seq; a.max_splits = max_splits; a.mode = mode;
+    a.ngrp = 1; a.ns = 2; a.tok_first = tok_first;
+    a.scale_log2 = p->scale * 1.4426950408889634f;
+    a.wait_cycles = (long long)dev.clock_khz * 2000LL;   // about two seconds of SM clocks
+
+    // first pass fixes the launch geometry (NG) without launching
+    int NG = 0;
+    rc = (p->head_dim == 128) ? dispatch_attn<128>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, true, &NG)
+                              : dispatch_attn<64>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, true, &NG);
+    if (rc != TS_OK) return rc;
+
+    const int chunks_per_group = env_int("TS_SPLIT_CHUNKS_PER_GROUP", 16);
+    ts_plan_kernel<<<1, 1024, 0, stream>>>(kv_lens, a.B, a.Hkv, NG, mode, max_splits, chunks_per_group,
+                                           reinterpret_cast<int32_t *>(ws + w.cum_tiles),
+                                           reinterpret_cast<GroupStart *>(ws + w.gstart),
+                                           reinterpret_cast<long long *>(ws + w.gpos), num_splits,
+                                           reinterpret_cast<int32_t *>(ws + w.status), a.part_o, a.part_lse,
+                                           p->q_len * p->num_q_heads, p->head_dim);
+    if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+
+    rc = (p->head_dim == 128) ? dispatch_attn<128>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, false, &NG)
+                              : dispatch_attn<64>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, false, &NG);
+    if (rc != TS_OK) return rc;
+
+    if (free_mode) {
+        const int pairs = a.B * a.Hkv;
+        if (p->head_dim == 128)
+            ts_merge_free_kernel<128><<<pairs, 128, 0, stream>>>(a.cum_tiles, a.part_o, a.part_lse, a.out, a.B, a.q_len,
+                                                                  a.Hq, a.Hkv, NG);
+        else
+            ts_merge_free_kernel<64><<<pairs, 128, 0, stream>>>(a.cum_tiles, a.part_o, a.part_lse, a.out, a.B, a.q_len,
+                                                                 a.Hq, a.Hkv, NG);
+        if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+    }
+    return TS_OK;
+}
+
+}  // namespace ts
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+size_t ts_attn_workspace_bytes(const ts_attn_params *p)
+{
+    if (ts::check_params(p) != TS_OK) return 0;
+    return ts::layout_workspace(p, true).total;
+}
+
+size_t ts_splitkv_workspace_bytes(const ts_attn_params *p)
+{
+    if (ts::check_params(p) != TS_OK) return 0;
+    return ts::layout_workspace(p, false).total;
+}
+
+int ts_decode_attn(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                   const int32_t *block_table, const int32_t *kv_lens, void *out, void *workspace,
+                   size_t workspace_bytes, void *stream)
+{
+    if (p && p->q_len != 1) return TS_ERR_INVALID_ARG;
+    return ts::run_attention(p, q, k_pool, v_pool, block_table, kv_lens, ts::kModeFree, 0, out, nullptr, nullptr,
+                             nullptr, workspace, workspace_bytes, stream);
+}
+
+int ts_verify_attn(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                   const int32_t *block_table, const int32_t *kv_lens, void *out, void *workspace,
+                   size_t workspace_bytes, void *stream)
+{
+    return ts::run_attention(p, q, k_pool, v_pool, block_table, kv_lens, ts::kModeFree, 0, out, nullptr, nullptr,
+                             nullptr, workspace, workspace_bytes, stream);
+}
+
+int ts_decode_attn_splitkv(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
+                           const int32_t *block_table, const int32_t *kv_lens, int32_t max_splits, float *partial_o,
+                           float *partial_lse, int32_t *num_splits, void *workspace, size_t workspace_bytes,
+                           void *stream)
+{
+    return ts::run_attention(p, q, k_pool, v_pool, block_table, kv_lens, ts::kModeChunks, max_splits, nullptr,
+                             partial_o, partial_lse, num_splits, workspace, workspace_bytes, stream);
+}
+
+int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *partial_o, const float *partial_lse,
+                 const int32_t *num_splits, void *out, void *stream)
+{
+    if (!p || !partial_o || !partial_lse || !num_splits || !out) return TS_ERR_INVALID_ARG;
+    if (p->num_seqs < 0 || p->q_len < 1 || p->num_q_heads < 1 || max_splits < 1) return TS_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return TS_ERR_UNSUPPORTED;
+    if (ts::misaligned(partial_o) || ts::misaligned(partial_lse) || ts::misaligned(num_splits) || ts::misaligned(out))
+        return TS_ERR_INVALID_ARG;
+    if (p->num_seqs == 0) return TS_OK;
+    const int rows_all = p->q_len * p->num_q_heads;
+    const long long rows = (long long)p->num_seqs * rows_all;
+    const unsigned grid = (unsigned)((rows + 3) / 4);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (p->head_dim == 128)
+        ts::ts_merge_dense_kernel<128><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,
+                                                             static_cast<uint16_t *>(out), p->num_seqs, rows_all, max_splits);
+    else
+        ts::ts_merge_dense_kernel<64><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,
+                                                            static_cast<uint16_t *>(out), p->num_seqs, rows_all, max_splits);
+    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
+const char *ts_status_string(int status)
+{
+    switch (status) {
+    case TS_OK: return "TS_OK";
+    case TS_ERR_INVALID_ARG: return "TS_ERR_INVALID_ARG";
+    case TS_ERR_UNSUPPORTED: return "TS_ERR_UNSUPPORTED";
+    case TS_ERR_WORKSPACE: return "TS_ERR_WORKSPACE";
+    case TS_ERR_CUDA: return "TS_ERR_CUDA";
+    case TS_ERR_TIMEOUT: return "TS_ERR_TIMEOUT";
+    default: return "TS_ERR_UNKNOWN";
+    }
+}
+
+}  // extern "C"
