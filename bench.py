@@ -1,0 +1,569 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-step hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
+
+One *step* is one pass of the whole hot path over the bulk-pool batch (256 sequences,
+lognormal KV lengths, 32/8 heads, head_dim 128, page 64): ``ts_decode_attn`` (planner,
+attention kernel, merge) followed by ``ts_accept_greedy`` with gamma = 0 (greedy
+selection of one token per sequence from bf16 logits ``[256, 1, 151936]``).  The
+headline value is decode tokens per second of that step with all inputs resident in
+HBM.  The same JSON line carries the roofline of the attention kernel, an end-to-end
+number with host buffers, the CPU oracle timed on this machine's host cores, clocks, and
+the other workloads (tail split-KV, speculative verify, mixed batch, concurrency sweep).
+
+``--impl reference`` times the CPU oracle (the only "reference" this method has: the
+paper ships no kernel) on the same workload and prints the same kind of line.
+With N > 1 (under torchrun) every rank runs its own replica of the batch (the path
+needs no collective); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_22788_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode_attn_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a timed region runs."""
+
+    REASONS = {
+        0x0000000000000004: "sw_power_cap",
+        0x0000000000000008: "hw_slowdown",
+        0x0000000000000020: "sw_thermal_slowdown",
+        0x0000000000000040: "hw_thermal_slowdown",
+        0x0000000000000080: "hw_power_brake_slowdown",
+    }
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.004):
+        self.samples, self.reasons, self.sm_max = [], set(), None
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.nv = pynvml
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["unavailable"], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.sm_max,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# device-side harness
+# ------------------------------------------------------------------------------------------------
+class Pool:
+    """One K pool and one V pool (HND layout) shared by every workload of a run."""
+
+    def __init__(self, num_pages: int, seed: int, num_kv_heads=8, page_size=64, head_dim=128, device=True):
+        import torch
+        self.num_pages, self.Hkv, self.P, self.D = num_pages, num_kv_heads, page_size, head_dim
+        shape = (num_pages, num_kv_heads, page_size, head_dim)
+        threads = os.cpu_count() or 8
+        self.k_host = wl.normal_bf16(shape, seed=seed * 1000 + 2, threads=threads)
+        self.v_host = wl.normal_bf16(shape, seed=seed * 1000 + 3, threads=threads)
+        if device:
+            self.k = torch.from_numpy(self.k_host.view(np.int16)).cuda().view(torch.bfloat16)
+            self.v = torch.from_numpy(self.v_host.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+class Workload:
+    """Block table, lengths and queries of one batch over the shared pool, on the device."""
+
+    def __init__(self, name, lens, pool: Pool, q_len=1, seed=0, Hq=32):
+        import torch
+        from paper_2608_22788_b200 import api
+        self.api = api
+        b = wl.make_batch(name, lens, q_len=q_len, num_q_heads=Hq, num_kv_heads=pool.Hkv, head_dim=pool.D,
+                          page_size=pool.P, seed=seed, layout="HND", fill=False)
+        assert b.num_pages <= pool.num_pages, (b.num_pages, pool.num_pages)
+        b.num_pages = pool.num_pages
+        b.q = wl.normal_bf16((b.num_seqs, q_len, Hq, pool.D), seed=seed * 1000 + 1)
+        self.b, self.pool = b, pool
+        self.geom = api.AttnGeometry(b.num_seqs, q_len, Hq, pool.Hkv, pool.D, pool.P, pool.num_pages,
+                                     b.max_pages_per_seq, b.kv_page_stride, b.kv_token_stride,
+                                     b.kv_head_stride, b.scale)
+        self.q = torch.from_numpy(b.q.view(np.int16)).cuda().view(torch.bfloat16)
+        self.bt = torch.from_numpy(b.block_table).cuda()
+        self.lens = torch.from_numpy(b.kv_lens).cuda()
+        self.out = torch.empty((b.num_seqs, q_len, Hq, pool.D), dtype=torch.bfloat16, device="cuda")
+        self.ws = torch.empty(api.attn_workspace_bytes(self.geom), dtype=torch.uint8, device="cuda")
+        self.bytes = b.algorithmic_bytes()
+
+    def attn(self):
+        f = self.api.ts_verify_attn if self.b.q_len > 1 else self.api.ts_decode_attn
+        f(self.geom, self.q, self.pool.k, self.pool.v, self.bt, self.lens, self.out, self.ws)
+
+    def status(self):
+        import torch
+        return int(self.ws[:4].view(torch.int32).item())
+
+
+class Accept:
+    def __init__(self, B, gamma, seed=0, vocab=wl.VOCAB):
+        import torch
+        from paper_2608_22788_b200 import api
+        self.api, self.B, self.gamma, self.V = api, B, gamma, vocab
+        self.logits_host = wl.make_logits(B, gamma, vocab, seed=seed, threads=os.cpu_count() or 8)
+        self.logits = torch.from_numpy(self.logits_host.view(np.int16)).cuda().view(torch.bfloat16)
+        self.draft = torch.zeros((B, max(gamma, 1)), dtype=torch.int32, device="cuda")[:, :gamma].contiguous()
+        self.tgt = torch.empty((B, gamma + 1), dtype=torch.int32, device="cuda")
+        self.acc = torch.empty((B,), dtype=torch.int32, device="cuda")
+        self.tok = torch.empty((B, gamma + 1), dtype=torch.int32, device="cuda")
+        self.ws = torch.empty(api.accept_workspace_bytes(B, gamma, vocab), dtype=torch.uint8, device="cuda")
+        self.bytes = B * (gamma + 1) * vocab * 2
+        if gamma > 0:          # drafts that follow the row maximum up to a seeded cut point
+            self.run()
+            torch.cuda.synchronize()
+            draft, self.cut = wl.make_draft(self.tgt.cpu().numpy(), vocab, seed=seed)
+            self.draft = torch.from_numpy(draft).cuda()
+
+    def run(self):
+        self.api.ts_accept_greedy(self.logits, self.draft if self.gamma > 0 else None, self.tgt, self.acc,
+                                  self.tok, self.ws)
+
+
+class L2Flusher:
+    def __init__(self, nbytes=512 << 20):
+        import torch
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+
+    def __call__(self):
+        self.buf.zero_()
+
+
+def time_with_flush(fn, flush, iters=7, warmup=3):
+    """Median / min milliseconds of ``fn`` with an L2 flush (untimed) before every call."""
+    import torch
+    for _ in range(warmup):
+        flush()
+        fn()
+    times = []
+    for _ in range(iters):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        times.append(a.elapsed_time(b))
+    return statistics.median(times), min(times)
+
+
+def gbs(nbytes, ms):
+    return nbytes / (ms * 1e-3) / 1e9
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm = the CPU oracle
+# ------------------------------------------------------------------------------------------------
+def oracle_step(oracle, b, logits_host, nseq, nthreads=0):
+    seqs = np.arange(nseq)
+    oracle.attention_batch(b, seqs=seqs, nthreads=nthreads)
+    oracle.accept_greedy(logits_host[:nseq], np.zeros((nseq, 0), np.int32), nthreads=nthreads)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    cores = oracle.max_threads()
+    lens = wl.lens_bulk(0)
+    b = wl.make_batch("bulk", lens, seed=0, threads=os.cpu_count() or 8)
+    logits = wl.make_logits(len(lens), 0, wl.VOCAB, seed=0, threads=os.cpu_count() or 8)
+    # calibrate on 16 sequences, then size the per-step sample so that the run stays short
+    t0 = time.perf_counter()
+    oracle_step(oracle, b, logits, 16)
+    per_tok = (time.perf_counter() - t0) / max(1, int(lens[:16].sum()))
+    budget = 90.0 / max(1, args.steps + args.warmup)
+    nseq = len(lens)
+    while nseq > 8 and per_tok * int(lens[:nseq].sum()) > budget:
+        nseq //= 2
+    for _ in range(args.warmup):
+        oracle_step(oracle, b, logits, nseq)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, b, logits, nseq)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = nseq / dt
+    sample = f"first {nseq} of 256 bulk sequences ({int(lens[:nseq].sum())} KV tokens) + their logits rows, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "bulk-pool decode step (256 seqs, lognormal KV lens, 32/8 heads, d128, page 64)"
+                               " + greedy token selection over [256,1,151936] logits", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_22788_b200 import api, build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: this library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0 and build.is_stale():
+        build.build()
+    if world > 1:
+        dist.barrier()
+    api.load_library()
+    peak, peak_src = measured_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    seed = rank
+    # ---- workloads over one shared pool
+    lens_bulk = wl.lens_bulk(seed)
+    specs = {"bulk": (lens_bulk, 1)}
+    if rank == 0 and not args.headline_only:
+        specs["tail"] = (wl.lens_tail(seed), 1)
+        for g in (4, 8, 16):
+            specs[f"verify_g{g}"] = (wl.lens_verify(seed), 1 + g)
+        specs["mixed"] = (wl.lens_mixed(seed), 1)
+    need_pages = 0
+    for lens, ql in specs.values():
+        need_pages = max(need_pages, wl.make_batch("x", lens, q_len=ql, fill=False).num_pages)
+    pool = Pool(need_pages, seed)
+    W = {name: Workload(name, lens, pool, q_len=ql, seed=seed) for name, (lens, ql) in specs.items()}
+    bulk = W["bulk"]
+    sampler_tokens = Accept(bulk.b.num_seqs, 0, seed=seed)
+
+    def step():
+        bulk.attn()
+        sampler_tokens.run()
+
+    # ---- headline: K back-to-back steps, inputs resident in HBM, KV (2.9 GB) >> L2
+    K, Wm = args.steps, max(3, args.warmup)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in ev:
+        a.record(); b.record()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(Wm):
+        step()
+    barrier()
+    with ClockSampler(local_rank) as clk:
+        start.record()
+        for i in range(K):
+            api.ts_set_attn_timing_events(ev[i][0], ev[i][1])
+            step()
+        stop.record()
+        torch.cuda.synchronize()
+    api.ts_set_attn_timing_events(None, None)
+    barrier()
+    assert bulk.status() == 0, "device status word reports a timed-out wait"
+    ms_total = start.elapsed_time(stop)
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / K
+    attn_ms = [a.elapsed_time(b) for a, b in ev]
+    attn_ms_avg = sum(attn_ms) / len(attn_ms)
+    tokens_per_step = bulk.b.num_seqs * world
+    value = tokens_per_step / (ms_step * 1e-3)
+    clocks = clk.summary()
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
+
+    achieved = gbs(bulk.bytes, attn_ms_avg)
+    roofline = {"bound": "hbm", "kernel": "ts_attn_kernel<128,1,1>", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "peak_source": peak_src, "algorithmic_bytes_per_launch": bulk.bytes,
+                "avg_launch_ms": attn_ms_avg, "traffic": args.ncu_traffic_bytes}
+
+    # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region
+    e2e = run_e2e(torch, api, bulk, sampler_tokens, pool, world)
+
+    # ---- CPU oracle on this machine's cores, same workload (a reported baseline, not the target)
+    cpu = run_cpu_baseline(bulk, pool, sampler_tokens)
+
+    extras = {}
+    if not args.headline_only:
+        extras = run_extras(torch, api, W, pool, peak, seed, quick=args.quick)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "bulk-pool decode step: 256 seqs/GPU, KV lens lognormal(median 2048, sigma 0.8) in "
+                               "[64,16384], 32 q / 8 kv heads, head_dim 128, page 64 (HND pool, permuted block table), "
+                               "q_len 1; then greedy token selection over bf16 logits [256,1,151936]",
+                   "step": "ts_decode_attn + ts_accept_greedy(gamma=0)", "kv_tokens_per_gpu": bulk.b.total_tokens,
+                   "l2": "inputs larger than L2 (KV %.2f GB per step vs 126 MB L2); no flush" % (bulk.bytes / 1e9),
+                   "parallelism": f"replicas x{world} (no collective on the path)", "seed": seed},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": 5 * K, "clocks": clocks,
+        "attn_only_tokens_per_s": bulk.b.num_seqs / (attn_ms_avg * 1e-3),
+        "workloads": extras,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def run_e2e(torch, api, bulk, sampler, pool, world):
+    """Same step, every input copied from pinned host memory and every result copied back, per step."""
+    K, Wm = 5, 3
+    host = {
+        "q": bulk.q.cpu().pin_memory(), "k": torch.from_numpy(pool.k_host.view(np.int16)).pin_memory(),
+        "v": torch.from_numpy(pool.v_host.view(np.int16)).pin_memory(), "bt": bulk.bt.cpu().pin_memory(),
+        "lens": bulk.lens.cpu().pin_memory(), "logits": sampler.logits.cpu().pin_memory(),
+    }
+    out_h = torch.empty(bulk.out.shape, dtype=torch.bfloat16).pin_memory()
+    tok_h = torch.empty(sampler.tok.shape, dtype=torch.int32).pin_memory()
+    k_i16, v_i16 = pool.k.view(torch.int16), pool.v.view(torch.int16)
+
+    def step(copy_kv: bool):
+        if copy_kv:
+            k_i16.copy_(host["k"], non_blocking=True)
+            v_i16.copy_(host["v"], non_blocking=True)
+        bulk.q.copy_(host["q"], non_blocking=True)
+        bulk.bt.copy_(host["bt"], non_blocking=True)
+        bulk.lens.copy_(host["lens"], non_blocking=True)
+        sampler.logits.copy_(host["logits"], non_blocking=True)
+        bulk.attn()
+        sampler.run()
+        out_h.copy_(bulk.out, non_blocking=True)
+        tok_h.copy_(sampler.tok, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    res = {}
+    for copy_kv in (True, False):
+        for _ in range(Wm):
+            step(copy_kv)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(K):
+            step(copy_kv)
+        torch.cuda.synchronize()
+        res[copy_kv] = (time.perf_counter() - t0) / K
+    nb = lambda t: t.numel() * t.element_size()
+    small = nb(host["q"]) + nb(host["bt"]) + nb(host["lens"]) + nb(host["logits"])
+    d2h = nb(out_h) + nb(tok_h)
+    B = bulk.b.num_seqs * world
+    return {"value": B / res[True], "unit": UNIT, "h2d_bytes_per_step": small + nb(host["k"]) + nb(host["v"]),
+            "d2h_bytes_per_step": d2h, "ms_per_step": res[True] * 1e3, "steps": K, "warmup": Wm,
+            "what": "every C-ABI input (q, K pool, V pool, block table, lengths, logits) copied from pinned host "
+                    "memory each step; outputs copied back",
+            "kv_cache_resident": {"value": B / res[False], "ms_per_step": res[False] * 1e3,
+                                  "h2d_bytes_per_step": small, "d2h_bytes_per_step": d2h,
+                                  "what": "same, with the KV cache kept in HBM between steps as a serving "
+                                          "engine does"}}
+
+
+def run_cpu_baseline(bulk, pool, sampler):
+    import oracle
+    b = bulk.b
+    b.k_pool, b.v_pool = pool.k_host, pool.v_host
+    cores = oracle.max_threads()
+    reps, t = 0, 0.0
+    while reps < 3 and t < 20.0:
+        t0 = time.perf_counter()
+        oracle_step(oracle, b, sampler.logits_host, b.num_seqs)
+        t += time.perf_counter() - t0
+        reps += 1
+    dt = t / reps
+    b.k_pool = b.v_pool = None
+    return {"value": b.num_seqs / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"the whole bulk batch ({b.num_seqs} seqs, {b.total_tokens} KV tokens) + its logits, "
+                      f"{reps} repetitions, {dt:.2f} s each", "ms_per_step": dt * 1e3}
+
+
+def run_extras(torch, api, W, pool, peak, seed, quick=False):
+    flush = L2Flusher()
+    out = {}
+
+    def record(name, nbytes, ms_med, ms_min, tokens, extra=None):
+        d = {"ms": ms_med, "ms_min": ms_min, "tokens_per_s": tokens / (ms_med * 1e-3), "GBps": gbs(nbytes, ms_med),
+             "frac_of_measured_peak": gbs(nbytes, ms_med) / peak, "frac_of_nominal_8TBs": gbs(nbytes, ms_med) / NOMINAL_HBM_GBS,
+             "algorithmic_bytes": nbytes}
+        if extra:
+            d.update(extra)
+        out[name] = d
+
+    for name in ("bulk", "tail", "mixed"):
+        w = W[name]
+        med, mn = time_with_flush(w.attn, flush)
+        record(name + ":ts_decode_attn", w.bytes, med, mn, w.b.num_seqs, {"kv_tokens": w.b.total_tokens})
+        assert w.status() == 0
+
+    # tail through the explicit split-KV entry point followed by the merge
+    w = W["tail"]
+    S = 256
+    po = torch.empty((w.b.num_seqs, S, 1, 32, 128), dtype=torch.float32, device="cuda")
+    pl = torch.empty((w.b.num_seqs, S, 1, 32), dtype=torch.float32, device="cuda")
+    ns = torch.empty((w.b.num_seqs,), dtype=torch.int32, device="cuda")
+    ws = torch.empty(api.splitkv_workspace_bytes(w.geom), dtype=torch.uint8, device="cuda")
+
+    def tail_split():
+        api.ts_decode_attn_splitkv(w.geom, w.q, pool.k, pool.v, w.bt, w.lens, S, po, pl, ns, ws)
+        api.ts_lse_merge(w.geom, S, po, pl, ns, w.out)
+
+    med, mn = time_with_flush(tail_split, flush)
+    record("tail:ts_decode_attn_splitkv+ts_lse_merge", w.bytes, med, mn, w.b.num_seqs,
+           {"max_splits": S, "num_splits": ns.cpu().tolist()})
+
+    # speculative verify: attention, then greedy acceptance
+    for g in (4, 8, 16):
+        w = W[f"verify_g{g}"]
+        acc = Accept(w.b.num_seqs, g, seed=seed)
+        med, mn = time_with_flush(w.attn, flush)
+        amed, amn = time_with_flush(acc.run, flush)
+        emitted = int((acc.acc + 1).sum().item())
+        assert w.status() == 0
+        record(f"verify_g{g}:ts_verify_attn", w.bytes, med, mn, w.b.num_seqs * (1 + g),
+               {"kv_tokens": w.b.total_tokens, "unit_note": "tokens_per_s counts scored positions B*(1+gamma)"})
+        record(f"verify_g{g}:ts_accept_greedy", acc.bytes, amed, amn, emitted,
+               {"emitted_tokens": emitted, "accepted_equals_seeded_cuts": bool((acc.acc.cpu().numpy() == acc.cut).all())})
+        out[f"verify_g{g}:emitted_tokens_per_s"] = emitted / ((med + amed) * 1e-3)
+        del acc
+
+    # concurrency sweep on the mixed length pool: attention-only analogue of v(b) and b*v(b)
+    pool_lens = wl.lens_mixed(seed)
+    sweep = {}
+    for c in (1, 4, 16, 64, 256, 1024):
+        draws = 1 if c == 1024 else (2 if quick else (5 if c <= 64 else 3))
+        rows = []
+        for dr in range(draws):
+            lens = pool_lens if c == 1024 else wl.sweep_subset(pool_lens, c, dr, seed)
+            sw = Workload(f"sweep{c}", lens, pool, seed=seed + 100 + dr)
+            med, mn = time_with_flush(sw.attn, flush, iters=5, warmup=2)
+            rows.append((c / (med * 1e-3), gbs(sw.bytes, med), med, int(lens.sum())))
+            del sw
+        tps = sorted(r[0] for r in rows)
+        sweep[str(c)] = {"tokens_per_s_median": statistics.median(tps), "tokens_per_s_min": tps[0],
+                         "tokens_per_s_max": tps[-1], "per_request_tokens_per_s": statistics.median(tps) / c,
+                         "GBps_median": statistics.median(r[1] for r in rows),
+                         "ms_median": statistics.median(r[2] for r in rows),
+                         "kv_tokens": [r[3] for r in rows], "draws": draws}
+    out["concurrency_sweep:ts_decode_attn"] = sweep
+
+    # the mixed batch as one uniform call versus a bulk call plus a tail call (lengths >= 16k to the tail)
+    lens = pool_lens
+    wb = Workload("mixed_bulk", lens[lens < 16384], pool, seed=seed + 7)
+    wt_lens = lens[lens >= 16384]
+    if len(wt_lens) > 0:
+        wt = Workload("mixed_tail", wt_lens, pool, seed=seed + 8)
+        mb, _ = time_with_flush(wb.attn, flush)
+        mt, _ = time_with_flush(wt.attn, flush)
+        out["mixed:split_into_bulk_and_tail_calls"] = {"bulk_ms": mb, "tail_ms": mt, "sum_ms": mb + mt,
+                                                       "uniform_ms": out["mixed:ts_decode_attn"]["ms"],
+                                                       "tail_seqs": int(len(wt_lens))}
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="fewer sweep draws")
+    ap.add_argument("--headline-only", action="store_true", help="skip the extra workloads")
+    ap.add_argument("--ncu-traffic-bytes", type=float, default=None,
+                    help="dram bytes per launch of the attention kernel from an ncu capture (reported as roofline.traffic)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

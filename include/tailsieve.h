@@ -160,6 +160,15 @@ int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draf
                      int32_t gamma, int32_t vocab, int32_t *target_argmax, int32_t *accept_len,
                      int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Instrumentation for benchmarks (the paper has no counterpart).  While both events (cudaEvent_t
+ * passed as void*) are non-NULL, every ts_decode_attn / ts_verify_attn / ts_decode_attn_splitkv
+ * call records `start_event` on its stream right before its attention kernel (after the planner)
+ * and `stop_event` right after it (before the merge).  Pass NULLs to switch it off.  Process-wide
+ * and not thread-safe.  Always returns TS_OK.
+ */
+int ts_set_attn_timing_events(void *start_event, void *stop_event);
+
 /* Static, human-readable name of a status code. */
 const char *ts_status_string(int status);
 

@@ -22,7 +22,7 @@ TS_OK = 0
 EXPORTED_SYMBOLS = (
     "ts_attn_workspace_bytes", "ts_splitkv_workspace_bytes", "ts_decode_attn", "ts_verify_attn",
     "ts_decode_attn_splitkv", "ts_lse_merge", "ts_accept_workspace_bytes", "ts_accept_greedy",
-    "ts_status_string",
+    "ts_set_attn_timing_events", "ts_status_string",
 )
 
 
@@ -70,6 +70,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ts_accept_workspace_bytes.argtypes = [i32, i32, i32]
     lib.ts_accept_greedy.restype = ctypes.c_int
     lib.ts_accept_greedy.argtypes = [vp, i64, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    lib.ts_set_attn_timing_events.restype = ctypes.c_int
+    lib.ts_set_attn_timing_events.argtypes = [vp, vp]
     lib.ts_status_string.restype = ctypes.c_char_p
     lib.ts_status_string.argtypes = [ctypes.c_int]
     if path == LIB_PATH:
@@ -193,3 +195,15 @@ def ts_accept_greedy(logits, draft, target_argmax, accept_len, out_tokens, works
                               workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "ts_accept_greedy")
     return target_argmax, accept_len, out_tokens
+
+
+def ts_set_attn_timing_events(start_event: Optional[torch.cuda.Event], stop_event: Optional[torch.cuda.Event]) -> None:
+    """Have later attention calls record the two events around their attention kernel (None = off).
+
+    The events must already exist on the device (``torch.cuda.Event(enable_timing=True)`` creates
+    its handle lazily: record it once before passing it here).
+    """
+    lib = load_library()
+    a = start_event.cuda_event if start_event is not None else None
+    b = stop_event.cuda_event if stop_event is not None else None
+    _check(lib.ts_set_attn_timing_events(a, b), "ts_set_attn_timing_events")

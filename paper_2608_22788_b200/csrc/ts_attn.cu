@@ -848,6 +848,8 @@ static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv,
     return TS_ERR_UNSUPPORTED;
 }
 
+static void *g_ev_start = nullptr, *g_ev_stop = nullptr;   // optional timing events (benchmarks)
+
 // Shared driver of the three attention entry points.
 static int run_attention(const ts_attn_params *p, const void *q, const void *k_pool, const void *v_pool,
                          const int32_t *block_table, const int32_t *kv_lens, int mode, int max_splits, void *out,
@@ -918,9 +920,11 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
                                            p->q_len * p->num_q_heads, p->head_dim);
     if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
 
+    if (g_ev_start && g_ev_stop) cudaEventRecord(static_cast<cudaEvent_t>(g_ev_start), stream);
     rc = (p->head_dim == 128) ? dispatch_attn<128>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, false, &NG)
                               : dispatch_attn<64>(a.rows, tk, tv, a, dev.sms, dev.smem_optin, stream, false, &NG);
     if (rc != TS_OK) return rc;
+    if (g_ev_start && g_ev_stop) cudaEventRecord(static_cast<cudaEvent_t>(g_ev_stop), stream);
 
     if (free_mode) {
         const int pairs = a.B * a.Hkv;
@@ -1000,6 +1004,13 @@ int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *parti
         ts::ts_merge_dense_kernel<64><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,
                                                             static_cast<uint16_t *>(out), p->num_seqs, rows_all, max_splits);
     return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
+int ts_set_attn_timing_events(void *start_event, void *stop_event)
+{
+    ts::g_ev_start = start_event;
+    ts::g_ev_stop = stop_event;
+    return TS_OK;
 }
 
 const char *ts_status_string(int status)

@@ -72,7 +72,13 @@ def normal_bf16(shape: Sequence[int], seed: int, std: float = 1.0, threads: int 
         x = rng.standard_normal(hi - lo, dtype=np.float32)
         if std != 1.0:
             x *= np.float32(std)
-        out[lo:hi] = f32_to_bf16_bits(x)
+        # same rounding as f32_to_bf16_bits, in place (the draws are finite, so no NaN branch)
+        u = x.view(np.uint32)
+        lsb = (u >> np.uint32(16)) & np.uint32(1)
+        u += lsb
+        u += np.uint32(0x7FFF)
+        u >>= np.uint32(16)
+        out[lo:hi] = u
 
     if nchunks == 1 or threads <= 1:
         for i in range(nchunks):
