@@ -161,6 +161,30 @@ int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draf
                      int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * ts_accept_greedy for callers that have no device memory to give and cannot get any.  (The paper
+ * has no counterpart; this is a packaging variant of ts_accept_greedy.)  Who that is: a serving
+ * process that handed all of HBM to its KV cache at start-up and kept no allocator for side
+ * buffers; a plug-in invoked from inside another framework's step, where calling cudaMalloc is
+ * off limits because it synchronises the whole device and may fail in an already full GPU; code
+ * that must not touch the allocator after initialisation.  Same arguments, results and error
+ * codes as ts_accept_greedy, minus the workspace: the chunk keys live in a 512 KB array that is
+ * part of the library image on every GPU that loads it (held until the process exits).
+ *   - Limit: num_seqs * (gamma + 1) <= 1024 rows; more returns TS_ERR_UNSUPPORTED and enqueues
+ *     nothing.  (16 sequences at gamma = 16 are 272 rows; 1024 decode sequences are 1024.)
+ *   - The call allocates nothing and frees nothing, on the host or the device.
+ *   - The first call on each device looks up the array's device address (a host-side query that
+ *     enqueues no work); make that first call before any stream capture is begun.
+ *   - All calls on one device share the array, which keeps whatever the previous call left in it.
+ *     Nothing in it has to be cleared between calls (each call overwrites every entry it later
+ *     reads), but two calls whose kernels may run at the same time on one GPU -- different streams,
+ *     or different host threads -- race on it and give wrong tokens: keep them on one stream or
+ *     order them yourself.
+ */
+int ts_accept_greedy_noalloc(const void *logits, int64_t row_stride, const int32_t *draft,
+                             int32_t num_seqs, int32_t gamma, int32_t vocab, int32_t *target_argmax,
+                             int32_t *accept_len, int32_t *out_tokens, void *stream);
+
+/*
  * Instrumentation for benchmarks (the paper has no counterpart).  While both events (cudaEvent_t
  * passed as void*) are non-NULL, every ts_decode_attn / ts_verify_attn / ts_decode_attn_splitkv
  * call records `start_event` on its stream right before its attention kernel (after the planner)

@@ -22,6 +22,7 @@ TS_OK = 0
 EXPORTED_SYMBOLS = (
     "ts_attn_workspace_bytes", "ts_splitkv_workspace_bytes", "ts_decode_attn", "ts_verify_attn",
     "ts_decode_attn_splitkv", "ts_lse_merge", "ts_accept_workspace_bytes", "ts_accept_greedy",
+    "ts_accept_greedy_noalloc",
     "ts_set_attn_timing_events", "ts_status_string",
 )
 
@@ -70,6 +71,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ts_accept_workspace_bytes.argtypes = [i32, i32, i32]
     lib.ts_accept_greedy.restype = ctypes.c_int
     lib.ts_accept_greedy.argtypes = [vp, i64, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    lib.ts_accept_greedy_noalloc.restype = ctypes.c_int
+    lib.ts_accept_greedy_noalloc.argtypes = [vp, i64, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.ts_set_attn_timing_events.restype = ctypes.c_int
     lib.ts_set_attn_timing_events.argtypes = [vp, vp]
     lib.ts_status_string.restype = ctypes.c_char_p
@@ -207,3 +210,22 @@ def ts_set_attn_timing_events(start_event: Optional[torch.cuda.Event], stop_even
     a = start_event.cuda_event if start_event is not None else None
     b = stop_event.cuda_event if stop_event is not None else None
     _check(lib.ts_set_attn_timing_events(a, b), "ts_set_attn_timing_events")
+
+
+def ts_accept_greedy_noalloc(logits, draft, target_argmax, accept_len, out_tokens, row_stride=None):
+    """``ts_accept_greedy`` for callers with no scratch to give: same results, no workspace argument.
+
+    The library keeps the intermediate keys in a fixed 512 KB device array of its own, so this call
+    works for at most 1024 rows (``B * (gamma + 1)``) and must not overlap on the GPU with another
+    call of itself (all calls on a device share that array).  Larger batches raise
+    ``TailSieveError`` (TS_ERR_UNSUPPORTED) without launching anything.
+    """
+    lib = load_library()
+    B, R, V = logits.shape
+    gamma = R - 1
+    stride = int(row_stride) if row_stride is not None else int(logits.stride(1))
+    rc = lib.ts_accept_greedy_noalloc(_ptr(logits, "logits"), stride, _ptr(draft, "draft") if gamma > 0 else None,
+                                      B, gamma, V, _ptr(target_argmax, "target_argmax"),
+                                      _ptr(accept_len, "accept_len"), _ptr(out_tokens, "out_tokens"), _stream())
+    _check(rc, "ts_accept_greedy_noalloc")
+    return target_argmax, accept_len, out_tokens

@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/tailsieve.h"
 
 namespace ts {
@@ -183,4 +185,68 @@ int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draf
     return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
+
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Acceptance without any caller-supplied or allocated scratch
+// ------------------------------------------------------------------------------------------------
+namespace ts {
+
+constexpr int kNoAllocMaxRows = 1024;   // num_seqs * (gamma + 1) accepted by ts_accept_greedy_noalloc
+
+// Chunk keys of ts_accept_greedy_noalloc: 1024 rows x 64 chunks x 8 B = 512 KB, resident on every
+// GPU that loads this library until the process exits.  Every call on a device shares it.
+static __device__ __align__(256) unsigned long long g_noalloc_keys[kNoAllocMaxRows * kMaxChunks];
+
+// Device address of g_noalloc_keys on the current device.  In host code the array's name is only a
+// handle for the runtime, not a device pointer, so the address is asked for once per device (with
+// that device current) and remembered.
+static int noalloc_keys_ptr(unsigned long long **out)
+{
+    static std::mutex mu;
+    static unsigned long long *cached[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TS_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev >= 0 && dev < 64 && cached[dev]) {
+        *out = cached[dev];
+        return TS_OK;
+    }
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_keys) != cudaSuccess || !p) return TS_ERR_CUDA;
+    if (dev >= 0 && dev < 64) cached[dev] = static_cast<unsigned long long *>(p);
+    *out = static_cast<unsigned long long *>(p);
+    return TS_OK;
+}
+
+}  // namespace ts
+
+extern "C" int ts_accept_greedy_noalloc(const void *logits, int64_t row_stride, const int32_t *draft,
+                                        int32_t num_seqs, int32_t gamma, int32_t vocab, int32_t *target_argmax,
+                                        int32_t *accept_len, int32_t *out_tokens, void *stream)
+{
+    if (num_seqs < 0 || gamma < 0 || vocab < 1) return TS_ERR_INVALID_ARG;
+    if (!logits || !target_argmax || !accept_len || !out_tokens) return TS_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft) return TS_ERR_INVALID_ARG;
+    if (row_stride < vocab) return TS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(logits) & 15u) return TS_ERR_INVALID_ARG;
+    const long long rows = (long long)num_seqs * (gamma + 1);
+    if (rows > ts::kNoAllocMaxRows) return TS_ERR_UNSUPPORTED;     // beyond the built-in scratch
+    if (rows == 0) return TS_OK;
+    unsigned long long *keys = nullptr;
+    const int rc = ts::noalloc_keys_ptr(&keys);
+    if (rc != TS_OK) return rc;
+    const int chunks = ts::pick_chunks(rows, vocab);
+    int chunk_len = (vocab + chunks - 1) / chunks;
+    chunk_len = (chunk_len + 7) / 8 * 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // every key this call reads in the second kernel is written by the first one, so nothing in the
+    // shared array has to start at zero
+    ts::ts_argmax_chunk_kernel<<<dim3((unsigned)chunks, (unsigned)rows), ts::kArgmaxThreads, 0, s>>>(
+        static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys);
+    if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+    ts::ts_accept_finish_kernel<<<1, 256, 0, s>>>(keys, chunks, draft, num_seqs, gamma, target_argmax, accept_len,
+                                                  out_tokens);
+    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
