@@ -549,6 +549,44 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
     return out
 
 
+def run_profile_case(args):
+    """A small, self-ending case of one kernel for profiler captures: inputs above the L2 size but
+    under 1 GB, three launches, no timing claims."""
+    import torch
+    from paper_2608_22788_b200 import api
+    torch.cuda.set_device(0)
+    api.load_library()
+    name = args.profile_case
+    if name == "bulk64":
+        lens, ql = wl.lens_bulk(0)[:64], 1
+    elif name == "tail2":
+        lens, ql = wl.lens_tail(0)[:2], 1
+    elif name.startswith("verify4_g"):
+        lens, ql = wl.lens_verify(0)[:4], 1 + int(name[len("verify4_g"):])
+    elif name.startswith("accept_g"):
+        g = int(name[len("accept_g"):])
+        acc = Accept(16, g, seed=0)
+        flush = L2Flusher(256 << 20)
+        for _ in range(3):
+            flush()
+            acc.run()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_case": name, "bytes": acc.bytes}))
+        return 0
+    else:
+        raise SystemExit(f"unknown profile case {name}")
+    pages = wl.make_batch("x", lens, q_len=ql, fill=False).num_pages
+    pool = Pool(pages, 0)
+    w = Workload(name, lens, pool, q_len=ql, seed=0)
+    for _ in range(3):
+        w.attn()
+    torch.cuda.synchronize()
+    assert w.status() == 0
+    print(json.dumps({"profile_case": name, "kv_tokens": w.b.total_tokens, "algorithmic_bytes": w.bytes,
+                      "units": w.b.num_seqs}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -559,7 +597,11 @@ def main():
     ap.add_argument("--headline-only", action="store_true", help="skip the extra workloads")
     ap.add_argument("--ncu-traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the attention kernel from an ncu capture (reported as roofline.traffic)")
+    ap.add_argument("--profile-case", default=None,
+                    help="run a small case for a profiler capture: bulk64, tail2, verify4_g4|8|16, accept_g4|8|16")
     args = ap.parse_args()
+    if args.profile_case:
+        return run_profile_case(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
