@@ -74,7 +74,7 @@ typedef struct ts_attn_params {
     float scale;               /* multiplies q.k in fp32, e.g. 1/sqrt(head_dim)                  */
 } ts_attn_params;
 
-/* Supported shapes: (num_q_heads / num_kv_heads) * q_len <= 96. */
+/* Supported shapes: (num_q_heads / num_kv_heads) * q_len <= 128 at head_dim 128, <= 96 at head_dim 64. */
 
 /*
  * Bytes of scratch that ts_decode_attn / ts_verify_attn need for `p` (depends on the head

@@ -565,6 +565,12 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     }
 }
 
+}  // namespace ts
+
+#include "ts_attn_tc.cuh"
+
+namespace ts {
+
 // ------------------------------------------------------------------------------------------------
 // merge kernels
 // ------------------------------------------------------------------------------------------------
@@ -737,7 +743,7 @@ static int check_params(const ts_attn_params *p)
     if (p->head_dim != 64 && p->head_dim != 128) return TS_ERR_UNSUPPORTED;
     if (p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128) return TS_ERR_UNSUPPORTED;
     const long long rows = (long long)(p->num_q_heads / p->num_kv_heads) * p->q_len;
-    if (rows > kMaxRows) return TS_ERR_UNSUPPORTED;
+    if (rows > (p->head_dim == 128 ? kMaxRowsD128 : kMaxRows)) return TS_ERR_UNSUPPORTED;
     if (!(p->scale == p->scale) || isinf(p->scale)) return TS_ERR_INVALID_ARG;
     return TS_OK;
 }
@@ -835,10 +841,37 @@ static int launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a
     return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
+// tcgen05 kernel: one CTA per SM, each CTA is one group of the tile line.
+static int launch_attn_tc(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a, int sms, int smem_optin,
+                          cudaStream_t stream, bool dry, int *ng_out)
+{
+    if ((size_t)smem_optin < tc::kSmemBytes) return TS_ERR_UNSUPPORTED;
+    int grid = sms;
+    const int grid_cap = env_int("TS_ATTN_GRID", 0);
+    if (grid_cap > 0 && grid_cap < grid) grid = grid_cap;
+    if (grid > kMaxGroups) grid = kMaxGroups;
+    *ng_out = grid;
+    a.ngrp = 1;
+    a.ns = tc::kStages;
+    if (dry) return TS_OK;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc::ts_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess)
+            return TS_ERR_CUDA;
+        attr_set = true;
+    }
+    tc::ts_attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tk, tv, a);
+    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
 template <int D>
 static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a, int sms, int smem_optin,
                          cudaStream_t stream, bool dry, int *ng)
 {
+    // more than one n-tile of rows at head_dim 128 and a positive scale: tcgen05 path
+    // (TS_ATTN_TC=0 keeps the warp-MMA path)
+    if (D == 128 && rows > 8 && rows <= 128 && a.scale_log2 > 0.f && env_int("TS_ATTN_TC", 1) != 0)
+        return launch_attn_tc(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 8) return launch_attn<D, 1, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 16) return launch_attn<D, 2, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 24) return launch_attn<D, 3, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);

@@ -9,7 +9,8 @@ namespace ts {
 
 constexpr int kTile = 64;          // KV tokens per pipeline stage
 constexpr int kMaxGroups = 1024;   // upper bound on warp groups in one launch (workspace sizing)
-constexpr int kMaxRows = 96;       // (Hq/Hkv) * q_len supported by the tiled kernels
+constexpr int kMaxRows = 96;       // (Hq/Hkv) * q_len supported by the warp-MMA kernels
+constexpr int kMaxRowsD128 = 128;  // ... and by the tcgen05 kernel (head_dim 128)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
