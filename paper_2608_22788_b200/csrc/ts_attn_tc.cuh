@@ -6,10 +6,11 @@
 //
 // One CTA per SM = one "group" of the planner's tile line.  Roles:
 //   warp 0      TMA producer: K/V tiles (64 tokens) into a 4-stage shared-memory ring
-//   warp 1      MMA issuer (one lane):  S[128 x 64]  = Q[128 x 128] . K^T     (8 x M128 N64 K16)
-//                                       O[128 x 128] += P[128 x 64] . V        (8 x M128 N128 K16,
-//                                                                               P as bf16 hi and lo)
-//   warps 2..5, 6..9  two softmax warpgroups, one thread per query row (TMEM lane) each; group w
+//   warp 1      first MMA issuer (one lane):   S[128 x 64]  = Q[128 x 128] . K^T   (8 x M128 N64 K16)
+//   warp 2      second MMA issuer (one lane):  O[128 x 128] += P[128 x 64] . V      (8 x M128 N128 K16,
+//               P as bf16 hi and lo).  Issuing one tcgen05.mma costs a thread 60-100 cycles here, more
+//               than these small MMAs take to execute, so the two kinds are issued by different threads.
+//   warps 3..6, 7..10  two softmax warpgroups, one thread per query row (TMEM lane) each; group w
 //               takes the tiles of parity w: S is read from TMEM, masked, exponentiated; each group
 //               has its own O accumulator in TMEM, kept there for the whole segment and rescaled
 //               only when a row's running maximum grows by more than 2^8 (lazy rescale), so the
@@ -24,13 +25,13 @@ namespace ts {
 namespace tc {
 
 constexpr int kStages = 6;
-constexpr int kThreads = 320;          // TMA warp, MMA warp, two softmax warpgroups of 4 warps
+constexpr int kThreads = 352;          // TMA warp, two MMA-issuing warps, two softmax warpgroups of 4 warps
 constexpr uint32_t kQBytes = 32768;          // 2 halves x 128 rows x 128 B
 constexpr uint32_t kStageBytes = 32768;      // K 16 KB + V 16 KB
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffStage = kOffQ + kQBytes;
 constexpr uint32_t kOffBar = kOffStage + kStages * kStageBytes;
-constexpr uint32_t kOffStats = kOffBar + 256;            // 128 x (m, l) of the second softmax warpgroup
+constexpr uint32_t kOffStats = kOffBar + 384;            // 128 x (m, l) of the second softmax warpgroup
 constexpr uint32_t kSmemBytes = kOffStats + 1024 + 1024;  // + alignment slack
 constexpr uint32_t kTmemCols = 512;          // four S/P buffers (64 each) + O0, O1 (128 each)
 constexpr uint32_t kTmemO = 256;             // first column of O0
@@ -141,6 +142,16 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int b_mn_major)
            ((uint32_t)(M >> 4) << 24);
 }
 
+// Optional phase timing of one softmax thread (CTA 0, first warp of each group): build with
+// -DTS_TC_TRACE; sums of SM clock cycles land in the 16 x 8-byte words after the status word.
+#ifdef TS_TC_TRACE
+#define TS_TRACE_DECL long long tr_t = clock64(), tr_acc[6] = {0, 0, 0, 0, 0, 0};
+#define TS_TRACE(i) { const long long tr_n = clock64(); tr_acc[i] += tr_n - tr_t; tr_t = tr_n; }
+#else
+#define TS_TRACE_DECL
+#define TS_TRACE(i)
+#endif
+
 struct Segment {
     int s, g, tau0, n, tiles, len, chunk_idx;
 };
@@ -182,7 +193,8 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     auto pfull = [&](int b) { return bsf + 8u * (4 + b); };      // per S/P buffer (4)
     auto obar = [&](int w) { return bsf + 8u * (8 + w); };       // per softmax group (2)
     const uint32_t qfull = bsf + 8u * 10;
-    const uint32_t tmem_slot = bsf + 8u * 11;
+    auto pdone = [&](int b) { return bsf + 8u * (11 + b); };     // per S/P buffer (4): its PV has finished
+    const uint32_t tmem_slot = bsf + 8u * 15;
 
     const GroupStart gs = a.gstart[gid];
     const int total = (int)(a.gpos[gid + 1] - a.gpos[gid]);
@@ -190,7 +202,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
     if (warp == 0 && lane == 0) {
         for (int st = 0; st < kStages; ++st) { mbar_init(kfull(st), 1); mbar_init(vfull(st), 1); mbar_init(kvfree(st), 1); }
-        for (int b = 0; b < 4; ++b) { mbar_init(sfull(b), 1); mbar_init(pfull(b), 4); }
+        for (int b = 0; b < 4; ++b) { mbar_init(sfull(b), 1); mbar_init(pfull(b), 4); mbar_init(pdone(b), 1); }
         for (int w = 0; w < 2; ++w) mbar_init(obar(w), 1);
         mbar_init(qfull, 4);
         mbar_fence_init();
@@ -242,9 +254,12 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
             return __shfl_sync(FULL, bt_cur, pg - bt_base);
         };
+        TS_TRACE_DECL
         for (int it = 0; it < total; ++it) {
             const int st = it % kStages;
+            TS_TRACE(0)
             if (it >= kStages) wait(kvfree(st), (uint32_t)(it / kStages - 1) & 1u);
+            TS_TRACE(1)
             const uint32_t kdst = base + kOffStage + (uint32_t)st * kStageBytes;
             const uint32_t vdst = kdst + 16384;
             int ids[4];
@@ -281,80 +296,115 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             cur_advance(ic, a);
         }
     } else if (warp == 1) {
-        // ============================================================ MMA issuer
+        // ============================================================ first MMA issuer: S = Q . K^T
         if (lane == 0) {
             constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0);
-            constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 1);
             const uint64_t dk = smem_desc_sw128(0, 16, 1024);          // K-major operands (Q, K tile)
-            const uint64_t dv = smem_desc_sw128(0, 8192, 1024);        // MN-major operand (V tile)
             const uint32_t q_lo = ((base + kOffQ) & 0x3ffffu) >> 4;
-            int it0 = 0, remaining = total, seg_no = 0;
-            // tile t uses S/P buffer 2*(t&1) + ((t>>1)&1); each buffer turns over every 4 tiles
-            auto issue_qk = [&](int t) {
-                const int st = t % kStages, buf = ((t & 1) << 1) | ((t >> 1) & 1);
-                wait(kfull(st), (uint32_t)(t / kStages) & 1u);
-                fence_after_sync();
-                const uint32_t k_lo = ((base + kOffStage + (uint32_t)st * kStageBytes) & 0x3ffffu) >> 4;
-                const uint32_t s_tmem = tmem_base + (uint32_t)buf * 64;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t ad = dk | (uint64_t)(q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2);
-                    const uint64_t bd = dk | (uint64_t)(k_lo + (kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
-                    umma_bf16(s_tmem, ad, bd, idesc_qk, kk == 0 ? 0u : 1u);
-                }
-                umma_commit(sfull(buf));
-            };
-            auto do_pv = [&](int t, bool first) {
-                const int st = t % kStages, w = t & 1, buf = (w << 1) | ((t >> 1) & 1);
-                wait(pfull(buf), (uint32_t)(t >> 2) & 1u);
-                wait(vfull(st), (uint32_t)(t / kStages) & 1u);
-                fence_after_sync();
-                const uint32_t p_tmem = tmem_base + (uint32_t)buf * 64;       // P overwrote S in place
-                const uint32_t v_lo = ((base + kOffStage + (uint32_t)st * kStageBytes + 16384) & 0x3ffffu) >> 4;
-                const uint32_t o_tmem = tmem_base + kTmemO + (uint32_t)w * 128;
-#pragma unroll
-                for (int part = 0; part < 2; ++part)          // hi (columns 0..31), then lo (32..63)
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t bd = dv | (uint64_t)(v_lo + ks * (2048 >> 4));
-                        umma_bf16_ts(o_tmem, p_tmem + part * 32 + ks * 8, bd, idesc_pv, (first && part == 0 && ks == 0) ? 0u : 1u);
-                    }
-                umma_commit(obar(w));
-                umma_commit(kvfree(st));
-            };
+            int t = 0, remaining = total, seg_no = 0, st = 0;
+            uint32_t st_par = 0;
+            TS_TRACE_DECL
             while (remaining > 0) {
                 const Segment sg = segment_at(cc, remaining, a);
                 wait(qfull, (uint32_t)seg_no & 1u);
-                fence_after_sync();
-                // scores run two tiles ahead of the second MMA, so both softmax groups always have work
-                for (int j = 0; j < sg.len; ++j) {
-                    issue_qk(it0 + j);
-                    if (j >= 2) do_pv(it0 + j - 2, j - 2 < 2);
+                for (int j = 0; j < sg.len; ++j, ++t) {
+                    // tile t uses S/P buffer 2*(t&1) + ((t>>1)&1); each buffer turns over every 4 tiles
+                    const int buf = ((t & 1) << 1) | ((t >> 1) & 1);
+                    TS_TRACE(0)
+                    if (t >= 4) wait(pdone(buf), (uint32_t)((t >> 2) - 1) & 1u);   // P of tile t-4 has been consumed
+                    wait(kfull(st), st_par);
+                    fence_after_sync();
+                    TS_TRACE(1)
+                    const uint32_t k_lo = ((base + kOffStage + (uint32_t)st * kStageBytes) & 0x3ffffu) >> 4;
+                    const uint32_t s_tmem = tmem_base + (uint32_t)buf * 64;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint64_t ad = dk | (uint64_t)(q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2);
+                        const uint64_t bd = dk | (uint64_t)(k_lo + (kk >> 2) * (8192 >> 4) + (kk & 3) * 2);
+                        umma_bf16(s_tmem, ad, bd, idesc_qk, kk == 0 ? 0u : 1u);
+                    }
+                    umma_commit(sfull(buf));
+                    TS_TRACE(2)
+                    if (++st == kStages) { st = 0; st_par ^= 1u; }
                 }
-                for (int j = sg.len >= 2 ? sg.len - 2 : 0; j < sg.len; ++j) do_pv(it0 + j, j < 2);
-                it0 += sg.len;
                 remaining -= sg.len;
                 cc.tau += sg.len - 1;
                 cur_advance(cc, a);
                 ++seg_no;
             }
+#ifdef TS_TC_TRACE
+            if (blockIdx.x == 0) {
+                long long *dbg = reinterpret_cast<long long *>(a.status) + 25;
+                for (int i = 0; i < 6; ++i) dbg[i] = tr_acc[i];
+                dbg[6] = total;
+            }
+#endif
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ============================================================ second MMA issuer: O += P . V
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 1);
+            const uint64_t dv = smem_desc_sw128(0, 8192, 1024);        // MN-major operand (V tile)
+            int t = 0, remaining = total, st = 0;
+            uint32_t st_par = 0;
+            TS_TRACE_DECL
+            while (remaining > 0) {
+                const Segment sg = segment_at(cc, remaining, a);
+                for (int j = 0; j < sg.len; ++j, ++t) {
+                    const int w = t & 1, buf = (w << 1) | ((t >> 1) & 1);
+                    TS_TRACE(0)
+                    wait(pfull(buf), (uint32_t)(t >> 2) & 1u);
+                    TS_TRACE(3)
+                    wait(vfull(st), st_par);
+                    fence_after_sync();
+                    TS_TRACE(4)
+                    const uint32_t p_tmem = tmem_base + (uint32_t)buf * 64;       // P overwrote S in place
+                    const uint32_t v_lo = ((base + kOffStage + (uint32_t)st * kStageBytes + 16384) & 0x3ffffu) >> 4;
+                    const uint32_t o_tmem = tmem_base + kTmemO + (uint32_t)w * 128;
+                    const bool first = j < 2;                 // tiles 0 and 1 of a segment start O0 / O1 afresh
+#pragma unroll
+                    for (int part = 0; part < 2; ++part)      // hi (columns 0..31), then lo (32..63)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t bd = dv | (uint64_t)(v_lo + ks * (2048 >> 4));
+                            umma_bf16_ts(o_tmem, p_tmem + part * 32 + ks * 8, bd, idesc_pv, (first && part == 0 && ks == 0) ? 0u : 1u);
+                        }
+                    umma_commit(pdone(buf));
+                    umma_commit(obar(w));
+                    umma_commit(kvfree(st));
+                    TS_TRACE(5)
+                    if (++st == kStages) { st = 0; st_par ^= 1u; }
+                }
+                remaining -= sg.len;
+                cc.tau += sg.len - 1;
+                cur_advance(cc, a);
+            }
+#ifdef TS_TC_TRACE
+            if (blockIdx.x == 0) {
+                long long *dbg = reinterpret_cast<long long *>(a.status) + 2 + 16;
+                for (int i = 0; i < 6; ++i) dbg[i] = tr_acc[i];
+                dbg[6] = total;
+            }
+#endif
         }
         __syncwarp();
     } else {
         // ============================================================ softmax warpgroups (one thread per row)
-        const int wg = (warp - 2) >> 2;                   // 0 or 1: parity of the tiles this group takes
+        const int wg = (warp - 3) >> 2;                   // 0 or 1: parity of the tiles this group takes
         const int q4 = warp & 3;
         const int row = q4 * 32 + lane;
         const uint32_t tlane = (uint32_t)(q4 * 32) << 16;
         const bool row_valid = row < a.rows;
         const int t_row = row_valid ? row / a.G : 0, hl = row_valid ? row % a.G : 0;
-        const int tid_wg = (threadIdx.x - 64) & 127;      // 0..127 inside the group
+        const int tid_wg = (threadIdx.x - 96) & 127;      // 0..127 inside the group
         const uint32_t o_col = kTmemO + (uint32_t)wg * 128u;
         const uint32_t stats = base + kOffStats + (uint32_t)row * 8u;
         // PV of tile t (parity wg) is the most recent commit on obar[wg] when this is called, so the
         // barrier is either in that phase or one past it: the parity test is unambiguous.
         auto wait_pv_done = [&](int t) { wait(obar(wg), (uint32_t)(t >> 1) & 1u); };
         int it0 = 0, remaining = total;
+        TS_TRACE_DECL
         while (remaining > 0) {
             const Segment sg = segment_at(cc, remaining, a);
             if (wg == 0) {
@@ -383,12 +433,15 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 last_t = it;
                 const int buf = (wg << 1) | ((it >> 1) & 1);
                 const uint32_t sp_tmem = tmem_base + tlane + (uint32_t)buf * 64;
+                TS_TRACE(0)
                 wait(sfull(buf), (uint32_t)(it >> 2) & 1u);
                 fence_after_sync();
+                TS_TRACE(1)
                 uint32_t xr[2][32];
                 tmem_ld32(sp_tmem, xr[0]);
                 tmem_ld32(sp_tmem + 32, xr[1]);
                 tmem_wait_ld();
+                TS_TRACE(2)
                 // mask (only near the sequence end) and row maximum of the raw scores (scale > 0 here)
                 const bool need_mask = tok0 + kTile - 1 > sg.n - a.q_len;
                 if (need_mask) {
@@ -414,6 +467,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 }
                 const float mref = (m_used == -INFINITY) ? 0.f : m_used;
                 // P = exp2(x - m) as bf16 hi + lo, written over S in TMEM: the A operand of the second MMA.
+                TS_TRACE(3)
                 float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -430,6 +484,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     tmem_st16(sp_tmem + 32 + 16 * h, lo);
                 }
                 const float rowsum = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                TS_TRACE(4)
                 // V rows past the sequence end may hold anything: zero them (0 * NaN)
                 const int valid_tok = sg.n - tok0;
                 if (valid_tok < kTile) {
@@ -464,6 +519,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pfull(buf));
                 l_sum = l_sum * alpha + rowsum;
+                TS_TRACE(5)
             }
             // ---- end of the segment: merge the two groups' accumulators, write the result
             if (last_t >= 0) wait_pv_done(last_t);
@@ -542,8 +598,18 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             cc.tau += sg.len - 1;
             cur_advance(cc, a);
         }
+#ifdef TS_TC_TRACE
+        if (blockIdx.x == 0 && q4 == 3 && lane == 0) {
+            long long *dbg = reinterpret_cast<long long *>(a.status) + 2 + 8 * wg;
+            for (int i = 0; i < 6; ++i) dbg[i] = tr_acc[i];
+            dbg[6] = total;
+        }
+#endif
     }
 
+#ifdef TS_TC_TRACE
+    // (written by the traced threads inside their branch; nothing to do here)
+#endif
     // ---- teardown
     fence_before_sync();
     __syncthreads();
