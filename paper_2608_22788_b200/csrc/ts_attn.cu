@@ -280,30 +280,33 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             tok_off = (ic.tau % tiles_per_page) * kTile;
         }
         if (lane == 0) {
-            const uint32_t bytes = (uint32_t)nbox * box_bytes * HALVES;
-            mbar_expect_tx(bk, bytes);
+            if (P >= kTile) {
+                // one instruction per tile and pool: box = 64 tokens x all halves
+                const uint32_t bytes = (uint32_t)TB;
+                mbar_expect_tx(bk, bytes);
+                tma_load_5d(kdst, &tmK, 0, tok_off, 0, ic.g, ids[0], bk);
+                mbar_expect_tx(bv, bytes);
+                tma_load_5d(vdst, &tmV, 0, tok_off, 0, ic.g, ids[0], bv);
+            } else {
+                const uint32_t bytes = (uint32_t)nbox * box_bytes * HALVES;
+                const int c1 = a.tok_first ? 0 : ic.g;
+                const int c2 = a.tok_first ? ic.g : 0;
+                mbar_expect_tx(bk, bytes);
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                if (b < nbox) {
+                for (int b = 0; b < 4; ++b)
+                    if (b < nbox) {
 #pragma unroll
-                    for (int h = 0; h < HALVES; ++h) {
-                        const int c1 = a.tok_first ? tok_off : ic.g;
-                        const int c2 = a.tok_first ? ic.g : tok_off;
-                        tma_load_4d(kdst + h * (kTile * 128) + b * box_bytes, &tmK, h * 64, c1, c2, ids[b], bk);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_4d(kdst + h * (kTile * 128) + b * box_bytes, &tmK, h * 64, c1, c2, ids[b], bk);
                     }
-                }
-            }
-            mbar_expect_tx(bv, bytes);
+                mbar_expect_tx(bv, bytes);
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                if (b < nbox) {
+                for (int b = 0; b < 4; ++b)
+                    if (b < nbox) {
 #pragma unroll
-                    for (int h = 0; h < HALVES; ++h) {
-                        const int c1 = a.tok_first ? tok_off : ic.g;
-                        const int c2 = a.tok_first ? ic.g : tok_off;
-                        tma_load_4d(vdst + h * (kTile * 128) + b * box_bytes, &tmV, h * 64, c1, c2, ids[b], bv);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_4d(vdst + h * (kTile * 128) + b * box_bytes, &tmV, h * 64, c1, c2, ids[b], bv);
                     }
-                }
             }
         }
     };
@@ -754,12 +757,29 @@ static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_para
 {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return TS_ERR_CUDA;
-    // dims: 0 = head_dim, then {token, head} by ascending stride, then page
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r;
+    if (p->page_size >= kTile) {
+        // 5-D: (64 dims, token, 64-dim half, head, page).  One box = 64 tokens x all halves, laid out in
+        // shared memory as [half][token][128 B]: a whole K or V tile per TMA instruction.
+        *tok_first = 1;
+        const cuuint64_t halves = (cuuint64_t)p->head_dim / 64;
+        cuuint64_t dims[5] = {64, (cuuint64_t)p->page_size, halves, (cuuint64_t)p->num_kv_heads, (cuuint64_t)p->num_pages};
+        cuuint64_t strides[4] = {(cuuint64_t)p->kv_token_stride * 2, 128, (cuuint64_t)p->kv_head_stride * 2,
+                                 (cuuint64_t)p->kv_page_stride * 2};
+        cuuint32_t box[5] = {64, (cuuint32_t)kTile, (cuuint32_t)halves, 1, 1};
+        r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(pool), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS ? TS_OK : TS_ERR_UNSUPPORTED;
+    }
+    // pages shorter than a tile: 4-D (64 dims, then {token, head} by ascending stride, page), one box
+    // per (page, half)
     const bool tf = p->kv_token_stride <= p->kv_head_stride;
     *tok_first = tf ? 1 : 0;
     cuuint64_t dims[4], strides[3];
-    cuuint32_t box[4], estr[4] = {1, 1, 1, 1};
-    const cuuint32_t box_tok = (cuuint32_t)(p->page_size < kTile ? p->page_size : kTile);
+    cuuint32_t box[4];
+    const cuuint32_t box_tok = (cuuint32_t)p->page_size;
     dims[0] = (cuuint64_t)p->head_dim;
     box[0] = 64;
     if (tf) {
@@ -770,9 +790,9 @@ static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_para
         dims[2] = (cuuint64_t)p->page_size; strides[1] = (cuuint64_t)p->kv_token_stride * 2; box[2] = box_tok;
     }
     dims[3] = (cuuint64_t)p->num_pages; strides[2] = (cuuint64_t)p->kv_page_stride * 2; box[3] = 1;
-    const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? TS_OK : TS_ERR_UNSUPPORTED;
 }
 

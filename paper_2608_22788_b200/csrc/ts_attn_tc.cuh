@@ -24,7 +24,10 @@
 namespace ts {
 namespace tc {
 
-constexpr int kStages = 6;
+#ifndef TS_TC_STAGES
+#define TS_TC_STAGES 6
+#endif
+constexpr int kStages = TS_TC_STAGES;
 constexpr int kThreads = 352;          // TMA warp, two MMA-issuing warps, two softmax warpgroups of 4 warps
 constexpr uint32_t kQBytes = 32768;          // 2 halves x 128 rows x 128 B
 constexpr uint32_t kStageBytes = 32768;      // K 16 KB + V 16 KB
@@ -145,11 +148,14 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int b_mn_major)
 // Optional phase timing of one softmax thread (CTA 0, first warp of each group): build with
 // -DTS_TC_TRACE; sums of SM clock cycles land in the 16 x 8-byte words after the status word.
 #ifdef TS_TC_TRACE
+// absolute timestamps of pipeline events of tiles 200..207 of CTA 0 (event e of tile t at ev[(t-200)*8 + e])
+#define TS_EVENT(t, e) { if (blockIdx.x == 0 && (t) >= 200 && (t) < 208) reinterpret_cast<long long *>(a.part_o)[((t) - 200) * 8 + (e)] = clock64(); }
 #define TS_TRACE_DECL long long tr_t = clock64(), tr_acc[6] = {0, 0, 0, 0, 0, 0};
 #define TS_TRACE(i) { const long long tr_n = clock64(); tr_acc[i] += tr_n - tr_t; tr_t = tr_n; }
 #else
+#define TS_EVENT(t, e) {}
 #define TS_TRACE_DECL
-#define TS_TRACE(i)
+#define TS_TRACE(i) {}
 #endif
 
 struct Segment {
@@ -230,15 +236,15 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
     if (warp == 0) {
         // ============================================================ TMA producer
+        // Kept free of integer divisions and long dependent chains: this warp has to issue one tile
+        // (4 tensor loads) every ~1000 cycles to stay ahead of the tensor pipe.
         Cursor ic = cc;
         int bt_s = -1, bt_base = 0, bt_cur = 0, bt_nxt = 0;
         const int P = a.P;
-        const int pages_per_tile = P < kTile ? kTile / P : 1;
-        const int tiles_per_page = P > kTile ? P / kTile : 1;
+        const int lgP = 31 - __clz(P);                    // page sizes are powers of two
         const int box_tok = P < kTile ? P : kTile;
         const uint32_t box_bytes = (uint32_t)box_tok * 128u;
-        auto page_id = [&](const Cursor &c, int pg) -> int {
-            const int npages = (c.n + P - 1) / P;
+        auto page_id = [&](const Cursor &c, int npages, int pg) -> int {
             const int32_t *row = a.block_table + (size_t)c.s * a.max_pages;
             if (c.s != bt_s || pg < bt_base || pg >= bt_base + 64) {
                 bt_s = c.s;
@@ -254,47 +260,68 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
             return __shfl_sync(FULL, bt_cur, pg - bt_base);
         };
+        int st = 0;
         TS_TRACE_DECL
+        uint32_t free_par = 0;                            // parity of the kvfree phase to wait for (from the 2nd lap on)
         for (int it = 0; it < total; ++it) {
-            const int st = it % kStages;
             TS_TRACE(0)
-            if (it >= kStages) wait(kvfree(st), (uint32_t)(it / kStages - 1) & 1u);
+            if (it >= kStages) wait(kvfree(st), free_par);
             TS_TRACE(1)
             const uint32_t kdst = base + kOffStage + (uint32_t)st * kStageBytes;
-            const uint32_t vdst = kdst + 16384;
+            const int npages = (ic.n + P - 1) >> lgP;
             int ids[4];
             int nbox = 1, tok_off = 0;
             if (P < kTile) {
-                const int first = ic.tau * pages_per_tile;
-                const int npages = (ic.n + P - 1) / P;
-                nbox = npages - first < pages_per_tile ? npages - first : pages_per_tile;
+                const int sh = 6 - lgP;                   // pages per tile = 1 << sh
+                const int first = ic.tau << sh;
+                nbox = npages - first < (1 << sh) ? npages - first : (1 << sh);
 #pragma unroll
-                for (int b = 0; b < 4; ++b) ids[b] = (b < nbox) ? page_id(ic, first + b) : 0;
+                for (int b = 0; b < 4; ++b) ids[b] = (b < nbox) ? page_id(ic, npages, first + b) : 0;
             } else {
-                ids[0] = page_id(ic, ic.tau / tiles_per_page);
-                tok_off = (ic.tau % tiles_per_page) * kTile;
+                const int sh = lgP - 6;                   // tiles per page = 1 << sh
+                ids[0] = page_id(ic, npages, ic.tau >> sh);
+                tok_off = (ic.tau & ((1 << sh) - 1)) << 6;
             }
+            TS_TRACE(2)
+            const uint32_t bytes = (P >= kTile) ? 16384u : (uint32_t)nbox * box_bytes * 2;
             if (lane == 0) {
-                const uint32_t bytes = (uint32_t)nbox * box_bytes * 2;
-                const int c1 = a.tok_first ? tok_off : ic.g;
-                const int c2 = a.tok_first ? ic.g : tok_off;
+                TS_EVENT(it, 7)
                 mbar_expect_tx(kfull(st), bytes);
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-                    if (b < nbox) {
-                        tma_load_4d(kdst + b * box_bytes, &tmK, 0, c1, c2, ids[b], kfull(st));
-                        tma_load_4d(kdst + 8192 + b * box_bytes, &tmK, 64, c1, c2, ids[b], kfull(st));
-                    }
                 mbar_expect_tx(vfull(st), bytes);
+            }
+            __syncwarp();
+            TS_TRACE(3)
+            if (P >= kTile) {
+                // lanes 0 and 1: one instruction per pool, a whole 64-token tile (both halves) each
+                if (lane < 2) {
+                    const void *tm = lane ? (const void *)&tmV : (const void *)&tmK;
+                    tma_load_5d(kdst + (lane ? 16384u : 0u), tm, 0, tok_off, 0, ic.g, ids[0], lane ? vfull(st) : kfull(st));
+                }
+            } else if (lane < 4) {
+                // short pages: lanes 0..3 = (K, dims 0-63), (K, 64-127), (V, 0-63), (V, 64-127), one box per page
+                const int c1 = a.tok_first ? 0 : ic.g;
+                const int c2 = a.tok_first ? ic.g : 0;
+                const bool is_v = lane >= 2;
+                const int h = lane & 1;
+                const void *tm = is_v ? (const void *)&tmV : (const void *)&tmK;
+                const uint32_t bar = is_v ? vfull(st) : kfull(st);
+                const uint32_t dst = kdst + (is_v ? 16384u : 0u) + (uint32_t)h * 8192u;
 #pragma unroll
                 for (int b = 0; b < 4; ++b)
-                    if (b < nbox) {
-                        tma_load_4d(vdst + b * box_bytes, &tmV, 0, c1, c2, ids[b], vfull(st));
-                        tma_load_4d(vdst + 8192 + b * box_bytes, &tmV, 64, c1, c2, ids[b], vfull(st));
-                    }
+                    if (b < nbox) tma_load_4d(dst + b * box_bytes, tm, h * 64, c1, c2, ids[b], bar);
             }
+            TS_TRACE(4)
             cur_advance(ic, a);
+            if (++st == kStages) { st = 0; if (it >= kStages) free_par ^= 1u; }
+            TS_TRACE(5)
         }
+#ifdef TS_TC_TRACE
+        if (blockIdx.x == 0 && lane == 0) {
+            long long *dbg = reinterpret_cast<long long *>(a.part_o) + 128;
+            for (int i = 0; i < 6; ++i) dbg[i] = tr_acc[i];
+            dbg[6] = total;
+        }
+#endif
     } else if (warp == 1) {
         // ============================================================ first MMA issuer: S = Q . K^T
         if (lane == 0) {
@@ -312,9 +339,11 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     const int buf = ((t & 1) << 1) | ((t >> 1) & 1);
                     TS_TRACE(0)
                     if (t >= 4) wait(pdone(buf), (uint32_t)((t >> 2) - 1) & 1u);   // P of tile t-4 has been consumed
+                    TS_EVENT(t, 2)
                     wait(kfull(st), st_par);
                     fence_after_sync();
                     TS_TRACE(1)
+                    TS_EVENT(t, 0)
                     const uint32_t k_lo = ((base + kOffStage + (uint32_t)st * kStageBytes) & 0x3ffffu) >> 4;
                     const uint32_t s_tmem = tmem_base + (uint32_t)buf * 64;
 #pragma unroll
@@ -325,6 +354,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     }
                     umma_commit(sfull(buf));
                     TS_TRACE(2)
+                    TS_EVENT(t, 1)
                     if (++st == kStages) { st = 0; st_par ^= 1u; }
                 }
                 remaining -= sg.len;
@@ -356,6 +386,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     TS_TRACE(0)
                     wait(pfull(buf), (uint32_t)(t >> 2) & 1u);
                     TS_TRACE(3)
+                    TS_EVENT(t, 5)
                     wait(vfull(st), st_par);
                     fence_after_sync();
                     TS_TRACE(4)
@@ -374,6 +405,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     umma_commit(obar(w));
                     umma_commit(kvfree(st));
                     TS_TRACE(5)
+                    TS_EVENT(t, 6)
                     if (++st == kStages) { st = 0; st_par ^= 1u; }
                 }
                 remaining -= sg.len;
@@ -400,8 +432,10 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const int tid_wg = (threadIdx.x - 96) & 127;      // 0..127 inside the group
         const uint32_t o_col = kTmemO + (uint32_t)wg * 128u;
         const uint32_t stats = base + kOffStats + (uint32_t)row * 8u;
-        // PV of tile t (parity wg) is the most recent commit on obar[wg] when this is called, so the
-        // barrier is either in that phase or one past it: the parity test is unambiguous.
+        // Wait until this group's PV of tile t (parity wg) has finished.  A parity wait only tells the
+        // current phase from the previous one, so every phase of obar[wg] is observed in order: the PV of
+        // tile it-2 before P of tile it is released (the PV of tile it cannot start earlier), and the PV
+        // of the group's last tile at the end of the segment.
         auto wait_pv_done = [&](int t) { wait(obar(wg), (uint32_t)(t >> 1) & 1u); };
         int it0 = 0, remaining = total;
         TS_TRACE_DECL
@@ -442,6 +476,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 tmem_ld32(sp_tmem + 32, xr[1]);
                 tmem_wait_ld();
                 TS_TRACE(2)
+                if (q4 == 3 && lane == 0) TS_EVENT(it, 3)
                 // mask (only near the sequence end) and row maximum of the raw scores (scale > 0 here)
                 const bool need_mask = tok0 + kTile - 1 > sg.n - a.q_len;
                 if (need_mask) {
@@ -496,11 +531,10 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 }
-                // lazy rescale of this group's O in TMEM (warp-collective): the PV of tile it-2, the last
-                // one that accumulated into it, must have finished (tile it-4's has: the scores of this
-                // tile were queued behind it)
+                // the PV of this group's previous tile (it-2), the last one that accumulated into its O
+                if (it >= 2) wait_pv_done(it - 2);
+                // lazy rescale of this group's O in TMEM (warp-collective)
                 if (__any_sync(FULL, rescale)) {
-                    wait_pv_done(it - 2);
                     fence_after_sync();
                     const float f = rescale ? alpha : 1.f;
 #pragma unroll 1
@@ -518,6 +552,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 if (valid_tok < kTile) fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pfull(buf));
+                if (q4 == 3 && lane == 0) TS_EVENT(it, 4)
                 l_sum = l_sum * alpha + rowsum;
                 TS_TRACE(5)
             }
