@@ -222,6 +222,7 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         tma_prefetch_desc(&tmV);
     }
     __syncthreads();
+    grid_dependency_wait();       // the planner's output is read from here on
 
     // ---- this group's piece of the tile line
     const GroupStart gs = a.gstart[gid];
@@ -609,17 +610,19 @@ __device__ __forceinline__ void merge_row(const float *po, size_t o_stride, cons
     }
 }
 
-// Free mode: one CTA (4 warps) per (s, g) pair; pairs covered by a single group are skipped.
+// Free mode: one warp per (s, g) pair, four pairs per CTA; pairs covered by a single group are skipped.
 template <int D>
 __global__ void __launch_bounds__(128)
 ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restrict__ part_o,
                      const float *__restrict__ part_lse, uint16_t *out, int B, int q_len, int Hq, int Hkv,
                      int NG)
 {
-    const int pair = blockIdx.x;
+    grid_dependency_wait();       // partials and direct outputs of the attention kernel
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pair = blockIdx.x * 4 + warp;
+    if (pair >= B * Hkv) return;
     const int s = pair / Hkv, g = pair % Hkv;
     const int G = Hq / Hkv, rows = G * q_len;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles = cum_tiles[s + 1] - cum_tiles[s];
     const long long W = (long long)Hkv * cum_tiles[B];
     int k_first = 0, k_last = -1;
@@ -629,7 +632,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restr
         k_last = (int)((b0 * NG - 1) / W);
         if (k_first == k_last) return;      // written directly by the attention kernel
     }
-    for (int r = warp; r < rows; r += 4) {
+    for (int r = 0; r < rows; ++r) {
         const int t = r / G, hl = r % G;
         uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
         if (tiles == 0) {
@@ -670,22 +673,76 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restr
     }
 }
 
-// Caller-visible dense layout: one warp per output row (s, t, h).
+// Caller-visible dense layout: one CTA (4 warps) per output row (s, t, h).  The splits of the row
+// are dealt round robin to the warps (lanes across head_dim), four loads in flight per warp; the
+// four partial sums are combined through shared memory.
 template <int D>
 __global__ void __launch_bounds__(128)
 ts_merge_dense_kernel(const float *__restrict__ part_o, const float *__restrict__ part_lse,
                       const int32_t *__restrict__ num_splits, uint16_t *out, int B, int rows_all, int max_splits)
 {
+    constexpr int V = D / 32;     // floats per lane
+    __shared__ float s_max[4];
+    __shared__ float s_w[4];
+    __shared__ float s_acc[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * 4 + warp;
-    if (row >= (long long)B * rows_all) return;
+    const long long row = blockIdx.x;
     const int s = (int)(row / rows_all), r = (int)(row % rows_all);
     int S = num_splits[s];
     if (S > max_splits) S = max_splits;
     if (S < 0) S = 0;
+    const size_t o_stride = (size_t)rows_all * D, l_stride = (size_t)rows_all;
     const float *po = part_o + ((size_t)s * max_splits * rows_all + r) * D;
     const float *pl = part_lse + (size_t)s * max_splits * rows_all + r;
-    merge_row<D>(po, (size_t)rows_all * D, pl, (size_t)rows_all, S, out + (size_t)row * D, lane);
+    // maximum of the log-sum-exps
+    float M = -INFINITY;
+    for (int i = threadIdx.x; i < S; i += 128) M = fmaxf(M, pl[(size_t)i * l_stride]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (lane == 0) s_max[warp] = M;
+    __syncthreads();
+    M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+    float acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = 0.f;
+    float Wsum = 0.f;
+    if (M != -INFINITY) {
+        for (int i0 = warp; i0 < S; i0 += 16) {
+            float w[4];
+            float x[4][V];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + 4 * u;
+                const float lse = i < S ? pl[(size_t)i * l_stride] : -INFINITY;
+                w[u] = lse == -INFINITY ? 0.f : expf(lse - M);
+                const float *p = po + (size_t)(i < S ? i : 0) * o_stride + lane * V;
+#pragma unroll
+                for (int v = 0; v < V; ++v) x[u][v] = w[u] != 0.f ? p[v] : 0.f;    // empty parts are not read into the sum
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                Wsum += w[u];
+#pragma unroll
+                for (int v = 0; v < V; ++v) acc[v] += w[u] * x[u][v];
+            }
+        }
+    }
+    if (lane == 0) s_w[warp] = Wsum;
+#pragma unroll
+    for (int v = 0; v < V; ++v) s_acc[warp][lane * V + v] = acc[v];
+    __syncthreads();
+    if (warp == 0) {
+        const float Wt = (s_w[0] + s_w[1]) + (s_w[2] + s_w[3]);
+        const float inv = Wt > 0.f ? 1.f / Wt : 0.f;
+        uint16_t *o = out + (size_t)row * D + lane * V;
+#pragma unroll
+        for (int v = 0; v < V; v += 2) {
+            const int d = lane * V + v;
+            const float a0 = (s_acc[0][d] + s_acc[1][d]) + (s_acc[2][d] + s_acc[3][d]);
+            const float a1 = (s_acc[0][d + 1] + s_acc[1][d + 1]) + (s_acc[2][d + 1] + s_acc[3][d + 1]);
+            *reinterpret_cast<uint32_t *>(o + v) = pack_bf16x2(a0 * inv, a1 * inv);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -857,8 +914,9 @@ static int launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a
             return TS_ERR_CUDA;
         attr_set = true;
     }
-    ts_attn_kernel<D, NT, WG><<<grid, ngrp * WG * 32, smem, stream>>>(tk, tv, a);
-    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+    const cudaError_t e = launch_overlapped(ts_attn_kernel<D, NT, WG>, dim3(grid), dim3(ngrp * WG * 32), smem, stream,
+                                            env_int("TS_PDL", 1) != 0, tk, tv, a);
+    return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
 // tcgen05 kernel: one CTA per SM, each CTA is one group of the tile line.
@@ -880,8 +938,9 @@ static int launch_attn_tc(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs
             return TS_ERR_CUDA;
         attr_set = true;
     }
-    tc::ts_attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tk, tv, a);
-    return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+    const cudaError_t e = launch_overlapped(tc::ts_attn_tc_kernel, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, stream,
+                                            env_int("TS_PDL", 1) != 0, tk, tv, a);
+    return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
 template <int D>
@@ -980,13 +1039,17 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     if (g_ev_start && g_ev_stop) cudaEventRecord(static_cast<cudaEvent_t>(g_ev_stop), stream);
 
     if (free_mode) {
+        const bool overlap = env_int("TS_PDL", 1) != 0;
         const int pairs = a.B * a.Hkv;
+        const dim3 mgrid((unsigned)((pairs + 3) / 4));
+        cudaError_t e;
         if (p->head_dim == 128)
-            ts_merge_free_kernel<128><<<pairs, 128, 0, stream>>>(a.cum_tiles, a.part_o, a.part_lse, a.out, a.B, a.q_len,
-                                                                  a.Hq, a.Hkv, NG);
+            e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles,
+                                  (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq, a.Hkv, NG);
         else
-            ts_merge_free_kernel<64><<<pairs, 128, 0, stream>>>(a.cum_tiles, a.part_o, a.part_lse, a.out, a.B, a.q_len,
-                                                                 a.Hq, a.Hkv, NG);
+            e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles,
+                                  (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq, a.Hkv, NG);
+        if (e != cudaSuccess) return TS_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
     }
     return TS_OK;
@@ -1048,7 +1111,8 @@ int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *parti
     if (p->num_seqs == 0) return TS_OK;
     const int rows_all = p->q_len * p->num_q_heads;
     const long long rows = (long long)p->num_seqs * rows_all;
-    const unsigned grid = (unsigned)((rows + 3) / 4);
+    if (rows > 0x7fffffffLL) return TS_ERR_UNSUPPORTED;
+    const unsigned grid = (unsigned)rows;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (p->head_dim == 128)
         ts::ts_merge_dense_kernel<128><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,

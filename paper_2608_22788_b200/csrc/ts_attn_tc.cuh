@@ -202,6 +202,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     auto pdone = [&](int b) { return bsf + 8u * (11 + b); };     // per S/P buffer (4): its PV has finished
     const uint32_t tmem_slot = bsf + 8u * 15;
 
+    grid_dependency_wait();      // the planner's output is read from here on
     const GroupStart gs = a.gstart[gid];
     const int total = (int)(a.gpos[gid + 1] - a.gpos[gid]);
     if (total <= 0) return;      // whole CTA leaves together, before anything is allocated

@@ -137,9 +137,35 @@ __device__ __forceinline__ float bf16hi_to_f32(uint32_t packed)
 {
     return __uint_as_float(packed & 0xffff0000u);
 }
+// Programmatic dependent launch: a kernel launched with the "programmatic stream serialization"
+// attribute may start while its predecessor in the stream is still running; it must execute this
+// before touching anything the predecessor writes (it returns once the predecessor has completed
+// and its writes are visible).  A no-op for a normally launched kernel.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Host helper: launch `kernel` allowing it to overlap the tail of the previous kernel in `stream`.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                            cudaStream_t stream, bool overlap, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 }  // namespace ts

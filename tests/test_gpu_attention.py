@@ -46,6 +46,10 @@ SHAPES = [
     ([513, 70, 1500, 17], 17, 32, 8, 128, 64, "HND"),         # rows 68 -> 3 warps
     ([700, 64, 24], 12, 16, 2, 128, 32, "NHD"),               # rows 96 -> 4 warps
     ([3, 700], 5, 4, 1, 64, 16, "HND"),                       # kv_len < q_len for seq 0
+    ([900, 64, 2500, 16], 16, 16, 2, 128, 64, "HND"),         # rows 128: the most the tcgen05 kernel takes
+    ([900, 33, 2500], 3, 32, 8, 128, 128, "NHD"),             # rows 12, page 128, token-major pool
+    ([900, 33, 2500], 9, 8, 2, 128, 16, "HND"),               # rows 36 with 16-token pages (4 boxes per tile)
+    ([2, 5000], 4, 8, 1, 128, 64, "HND"),                     # rows 32, a single kv head
 ]
 
 
@@ -209,3 +213,27 @@ def test_few_ctas_many_tiles_per_group(grid, ql, monkeypatch):
     assert_close(out, ref, f"grid={grid} ql={ql}")
     po, pl, ns = d.splitkv(5)
     assert_close(d.out, ref, f"splitkv grid={grid} ql={ql}")
+
+
+@pytest.mark.parametrize("scale", [-0.07, 0.0])
+def test_non_positive_scale_takes_the_warp_mma_path(scale):
+    # the tcgen05 kernel assumes scale > 0 (it takes row maxima of the raw scores); other scales
+    # are legal inputs and must still be exact
+    b = wl.make_batch("ns", [300, 1000, 77], q_len=5, num_q_heads=8, num_kv_heads=2, head_dim=128, page_size=64,
+                      seed=77, poison=True, scale=scale)
+    ref, _ = oracle.attention_batch(b)
+    assert_close(DeviceBatch(b).verify(), ref, f"scale={scale}")
+    b1 = wl.make_batch("ns", [300, 1000, 77], num_q_heads=8, num_kv_heads=2, head_dim=128, page_size=64,
+                       seed=78, poison=True, scale=scale)
+    ref1, _ = oracle.attention_batch(b1)
+    assert_close(DeviceBatch(b1).decode(), ref1, f"decode scale={scale}")
+
+
+def test_both_verify_kernels_agree_with_the_oracle(monkeypatch):
+    # same inputs through the tcgen05 kernel (default) and the warp-MMA kernel (TS_ATTN_TC=0)
+    b = wl.make_batch("two", [513, 70, 2300, 9], q_len=9, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                      page_size=64, seed=5, poison=True)
+    ref, _ = oracle.attention_batch(b)
+    assert_close(DeviceBatch(b).verify(), ref, "tcgen05")
+    monkeypatch.setenv("TS_ATTN_TC", "0")
+    assert_close(DeviceBatch(b).verify(), ref, "warp mma")
