@@ -39,6 +39,9 @@ METRIC = "decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, decode attention kernel, from the
+# ncu capture summarised in profiles/ts_attn_kernel_decode_bulk64.md (traffic grows with the KV bytes)
+NCU_TRAFFIC_RATIO_DECODE = 1.025
 
 
 def measured_peaks():
@@ -303,7 +306,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    seed = rank
+    from paper_2608_22788_b200 import replicas as _rep
+    seed = _rep.rank_seed(0, rank)
     # ---- workloads over one shared pool
     lens_bulk = wl.lens_bulk(seed)
     specs = {"bulk": (lens_bulk, 1)}
@@ -343,16 +347,13 @@ def run_ours(args):
     api.ts_set_attn_timing_events(None, None)
     barrier()
     assert bulk.status() == 0, "device status word reports a timed-out wait"
-    ms_total = start.elapsed_time(stop)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    from paper_2608_22788_b200 import replicas
+    dev = torch.device("cuda", local_rank)
+    value, tokens_per_step, ms_total = replicas.job_throughput(bulk.b.num_seqs * K, start.elapsed_time(stop), dev)
+    tokens_per_step /= K
     ms_step = ms_total / K
     attn_ms = [a.elapsed_time(b) for a, b in ev]
     attn_ms_avg = sum(attn_ms) / len(attn_ms)
-    tokens_per_step = bulk.b.num_seqs * world
-    value = tokens_per_step / (ms_step * 1e-3)
     clocks = clk.summary()
 
     if rank != 0:
@@ -362,10 +363,13 @@ def run_ours(args):
         return 0
 
     achieved = gbs(bulk.bytes, attn_ms_avg)
-    roofline = {"bound": "hbm", "kernel": "ts_attn_kernel<128,1,1>", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "peak_source": peak_src, "algorithmic_bytes_per_launch": bulk.bytes,
-                "avg_launch_ms": attn_ms_avg, "traffic": args.ncu_traffic_bytes}
+    traffic = args.ncu_traffic_bytes if args.ncu_traffic_bytes is not None else NCU_TRAFFIC_RATIO_DECODE * bulk.bytes
+    roofline = {"bound": "hbm", "kernel": "ts_attn_kernel<128,1,1> (decode attention, bulk batch)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": bulk.bytes, "avg_launch_ms": attn_ms_avg, "traffic": traffic,
+                "traffic_note": "dram read+write bytes of an ncu capture of the same kernel on the first 64 bulk "
+                                "sequences (profiles/ts_attn_kernel_decode_bulk64.md), scaled by algorithmic bytes"}
 
     # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region
     e2e = run_e2e(torch, api, bulk, sampler_tokens, pool, world)

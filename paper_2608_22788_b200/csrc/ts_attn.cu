@@ -610,7 +610,8 @@ __device__ __forceinline__ void merge_row(const float *po, size_t o_stride, cons
     }
 }
 
-// Free mode: one warp per (s, g) pair, four pairs per CTA; pairs covered by a single group are skipped.
+// Free mode: one CTA (4 warps, one output row each at a time) per (s, g) pair; pairs covered by a
+// single group are skipped.
 template <int D>
 __global__ void __launch_bounds__(128)
 ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restrict__ part_o,
@@ -619,8 +620,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restr
 {
     grid_dependency_wait();       // partials and direct outputs of the attention kernel
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = blockIdx.x * 4 + warp;
-    if (pair >= B * Hkv) return;
+    const int pair = blockIdx.x;
     const int s = pair / Hkv, g = pair % Hkv;
     const int G = Hq / Hkv, rows = G * q_len;
     const int tiles = cum_tiles[s + 1] - cum_tiles[s];
@@ -632,7 +632,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restr
         k_last = (int)((b0 * NG - 1) / W);
         if (k_first == k_last) return;      // written directly by the attention kernel
     }
-    for (int r = 0; r < rows; ++r) {
+    for (int r = warp; r < rows; r += 4) {
         const int t = r / G, hl = r % G;
         uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
         if (tiles == 0) {
@@ -1041,7 +1041,7 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     if (free_mode) {
         const bool overlap = env_int("TS_PDL", 1) != 0;
         const int pairs = a.B * a.Hkv;
-        const dim3 mgrid((unsigned)((pairs + 3) / 4));
+        const dim3 mgrid((unsigned)pairs);
         cudaError_t e;
         if (p->head_dim == 128)
             e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles,
