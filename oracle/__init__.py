@@ -56,6 +56,10 @@ def _load():
         lib.ora_accept_greedy.restype = ctypes.c_int
         lib.ora_accept_greedy.argtypes = [c_u16p, ctypes.c_int64, c_i32p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_int, c_i32p, c_i32p, c_i32p, ctypes.c_int]
+        lib.ora_accept_sample.restype = ctypes.c_int
+        lib.ora_accept_sample.argtypes = [c_u16p, ctypes.c_int64, c_i32p, c_f64p, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
+                                          c_i32p, c_i32p, c_i32p, c_f64p]
         lib.ora_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -150,3 +154,29 @@ def accept_greedy(logits, draft, nthreads: int = 0):
     if rc != 0:
         raise RuntimeError(f"ora_accept_greedy failed ({rc})")
     return tgt, acc, out
+
+
+def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, top_p: float):
+    """Lossless acceptance under temperature / top-k / top-p sampling with point-proposal drafts.
+
+    ``logits``: uint16 bf16 bits ``[B, gamma+1, V]``; ``draft``: int ``[B, gamma]``; ``uniforms``:
+    float ``[B, gamma+1, 2]`` in [0, 1).  Returns ``(accept_len [B], out_tokens [B,gamma+1],
+    kept_ids [B,gamma+1,top_k], kept_p [B,gamma+1,top_k])``.
+    """
+    lib = _load()
+    logits = np.ascontiguousarray(logits, dtype=np.uint16)
+    B, R, V = logits.shape
+    gamma = R - 1
+    draft = np.ascontiguousarray(draft, dtype=np.int32).reshape(B, gamma)
+    u = np.ascontiguousarray(uniforms, dtype=np.float64).reshape(B, R, 2)
+    acc = np.empty((B,), dtype=np.int32)
+    out = np.empty((B, R), dtype=np.int32)
+    ids = np.empty((B, R, top_k), dtype=np.int32)
+    pp = np.empty((B, R, top_k), dtype=np.float64)
+    rc = lib.ora_accept_sample(_p(logits, ctypes.c_uint16), V, _p(draft, ctypes.c_int32), _p(u, ctypes.c_double),
+                               B, gamma, V, float(temperature), int(top_k), float(top_p),
+                               _p(acc, ctypes.c_int32), _p(out, ctypes.c_int32), _p(ids, ctypes.c_int32),
+                               _p(pp, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ora_accept_sample failed ({rc})")
+    return acc, out, ids, pp

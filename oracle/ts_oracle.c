@@ -24,6 +24,9 @@
  *                        (Section 3.4): per-row lowest-index argmax over the
  *                        vocabulary, then the longest draft prefix that agrees
  *                        with it, plus one token from the target.
+ *   ora_accept_sample    the same verification under the paper's sampling
+ *                        regime (temperature, top-k, top-p; Appendix, Table
+ *                        "shared-sampling-config") with point-proposal drafts.
  *
  * All bf16 inputs are uint16 bit patterns, decoded exactly to double.
  * Pins for every function live in tests/test_oracle_*.py (brute force on
@@ -222,4 +225,100 @@ int ora_max_threads(void)
 #else
     return 1;
 #endif
+}
+
+/*
+ * Lossless acceptance of a draft block under temperature / top-k / top-p sampling -- the paper's
+ * rollout sampling regime (Appendix, Table "shared-sampling-config": temperature 0.7, top-p 0.8,
+ * top-k 20) combined with the speculative-sampling rule it adopts (Section 3.4, lossless
+ * formulation).  The draft proposes ONE token per position (a point proposal, as greedy MTP-style
+ * drafters do), i.e. the draft distribution is q = one-hot(draft token).
+ *
+ * For every row (b, i), i in [0, gamma]:
+ *   1. candidates = the top_k largest logits; equal logits are ordered by ascending index
+ *      (numeric comparison: +0 == -0); NaN logits are never candidates
+ *   2. z_j = logit_j / temperature, p_j = exp(z_j - z_max) / sum over the candidates
+ *   3. nucleus: keep the shortest prefix (in the order of step 1) whose probabilities sum to
+ *      at least top_p (always at least one token); renormalise over the kept tokens
+ * Acceptance for sequence b walks i = 0 .. gamma-1 with the uniforms u[b, i, 0] (accept) and
+ * u[b, i, 1] (resample), all in [0, 1):
+ *   - draft token x accepted iff x is kept and u_accept < p(x)
+ *   - on rejection emit y drawn from norm(max(0, p - q)) = p restricted to the kept tokens other
+ *     than x, by inverse CDF over the kept order: first j with cumulative weight > u_sample * total;
+ *     stop
+ *   - if all gamma drafts are accepted, emit one more token drawn from p_gamma the same way
+ *     (nothing removed)
+ * out_tokens = accepted drafts ++ that one token, padded with -1; accept_len = number accepted.
+ *
+ * The probabilities of every row are also returned (kept_ids / kept_p, top_k slots per row, -1 / 0
+ * padded) so that tests can tell a wrong decision from one where u falls within rounding of p.
+ */
+int ora_accept_sample(const uint16_t *logits, int64_t row_stride, const int32_t *draft,
+                      const double *uniforms /* [B, gamma+1, 2] */, int B, int gamma, int V,
+                      double temperature, int top_k, double top_p, int32_t *accept_len,
+                      int32_t *out_tokens, int32_t *kept_ids /* [B, gamma+1, top_k] */,
+                      double *kept_p /* [B, gamma+1, top_k] */)
+{
+    if (B < 0 || gamma < 0 || V <= 0 || top_k < 1 || !(temperature > 0.0)) return -1;
+    const int R = gamma + 1;
+    for (int r = 0; r < B * R; ++r) {
+        const uint16_t *row = logits + (int64_t)r * row_stride;
+        int32_t *ids = kept_ids + (int64_t)r * top_k;
+        double *pp = kept_p + (int64_t)r * top_k;
+        double val[top_k];
+        int n = 0;
+        /* step 1: insertion into a list sorted by (value descending, index ascending) */
+        for (int v = 0; v < V; ++v) {
+            const double x = bf16_to_double(row[v]);
+            if (x != x) continue;                       /* NaN */
+            if (n == top_k && !(x > val[n - 1])) continue;   /* not better than the worst kept (ties lose: higher index) */
+            int pos = n < top_k ? n : top_k - 1;
+            while (pos > 0 && x > val[pos - 1]) { val[pos] = val[pos - 1]; ids[pos] = ids[pos - 1]; --pos; }
+            val[pos] = x; ids[pos] = v;
+            if (n < top_k) ++n;
+        }
+        /* steps 2 and 3 */
+        double sum = 0.0;
+        for (int j = 0; j < n; ++j) { pp[j] = exp(val[j] / temperature - val[0] / temperature); sum += pp[j]; }
+        int keep = 0;
+        double cum = 0.0;
+        for (int j = 0; j < n; ++j) { pp[j] /= sum; }
+        for (int j = 0; j < n; ++j) { cum += pp[j]; keep = j + 1; if (cum >= top_p) break; }
+        double ksum = 0.0;
+        for (int j = 0; j < keep; ++j) ksum += pp[j];
+        for (int j = 0; j < keep; ++j) pp[j] /= ksum;
+        for (int j = keep; j < top_k; ++j) { ids[j] = -1; pp[j] = 0.0; }
+    }
+    for (int b = 0; b < B; ++b) {
+        int32_t *out = out_tokens + (int64_t)b * R;
+        for (int i = 0; i < R; ++i) out[i] = -1;
+        int a = 0;
+        for (int i = 0; i <= gamma; ++i) {
+            const int32_t *ids = kept_ids + ((int64_t)b * R + i) * top_k;
+            const double *pp = kept_p + ((int64_t)b * R + i) * top_k;
+            const double ua = uniforms[((int64_t)b * R + i) * 2], us = uniforms[((int64_t)b * R + i) * 2 + 1];
+            int skip = -1;                 /* slot of the rejected draft token, if any */
+            if (i < gamma) {
+                const int32_t x = draft[(int64_t)b * gamma + i];
+                double px = 0.0;
+                for (int j = 0; j < top_k; ++j) if (ids[j] == x) { px = pp[j]; skip = j; }
+                if (ua < px) { out[i] = x; ++a; continue; }
+            }
+            /* emit one token from the (residual) distribution and stop */
+            double total = 0.0;
+            for (int j = 0; j < top_k; ++j) if (ids[j] >= 0 && j != skip) total += pp[j];
+            double cum = 0.0;
+            int32_t y = -1;
+            for (int j = 0; j < top_k; ++j) {
+                if (ids[j] < 0 || j == skip) continue;
+                cum += pp[j];
+                y = ids[j];
+                if (cum > us * total) break;
+            }
+            out[i] = y;
+            break;
+        }
+        accept_len[b] = a;
+    }
+    return 0;
 }

@@ -1,0 +1,151 @@
+"""Pins for the oracle's stochastic (temperature / top-k / top-p) lossless acceptance (CPU only)."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_22788_b200 import workloads as wl
+
+
+def _bits(x):
+    return wl.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+def filtered_distribution(row_f64, temperature, top_k, top_p):
+    """Independent NumPy version of steps 1-3: returns (ids in order, probabilities)."""
+    v = np.asarray(row_f64, np.float64)
+    idx = np.arange(len(v))
+    ok = ~np.isnan(v)
+    order = sorted(idx[ok], key=lambda i: (-v[i], i))[:top_k]
+    z = np.array([v[i] for i in order]) / temperature
+    p = np.exp(z - z.max()) if len(z) else z
+    p = p / p.sum() if len(z) else p
+    keep = int(np.searchsorted(np.cumsum(p), top_p - 1e-300, side="left")) + 1 if len(p) else 0
+    keep = min(keep, len(p))
+    p = p[:keep] / p[:keep].sum() if keep else p[:0]
+    return list(order[:keep]), p
+
+
+def brute_accept(logits_bits, draft, u, temperature, top_k, top_p):
+    f = wl.bf16_bits_to_f32(logits_bits).astype(np.float64)
+    B, R, V = f.shape
+    gamma = R - 1
+    acc = np.zeros(B, np.int32)
+    out = np.full((B, R), -1, np.int32)
+    for b in range(B):
+        for i in range(R):
+            ids, p = filtered_distribution(f[b, i], temperature, top_k, top_p)
+            if i < gamma:
+                x = int(draft[b, i])
+                px = p[ids.index(x)] if x in ids else 0.0
+                if u[b, i, 0] < px:
+                    out[b, i] = x
+                    acc[b] += 1
+                    continue
+                rest = [(t, q) for t, q in zip(ids, p) if t != x]
+            else:
+                rest = list(zip(ids, p))
+            total = sum(q for _, q in rest)
+            cum, y = 0.0, -1
+            for t, q in rest:
+                cum += q
+                y = t
+                if cum > u[b, i, 1] * total:
+                    break
+            out[b, i] = y
+            break
+    return acc, out
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_matches_numpy_bruteforce(seed):
+    rng = np.random.default_rng(seed)
+    B, gamma, V = 5, 4, 200
+    logits = wl.make_logits(B, gamma, V, seed=seed)
+    best = np.argmax(wl.bf16_bits_to_f32(logits), -1)
+    draft = np.where(rng.random((B, gamma)) < 0.7, best[:, :gamma], rng.integers(0, V, (B, gamma))).astype(np.int32)
+    u = rng.random((B, gamma + 1, 2))
+    T, k, pnuc = [(0.7, 20, 0.8), (1.0, 5, 0.95), (0.3, 20, 1.0), (2.0, 50, 0.5), (0.7, 1, 0.8), (0.7, 20, 0.8)][seed]
+    acc, out, ids, pp = oracle.accept_sample(logits, draft, u, temperature=T, top_k=k, top_p=pnuc)
+    racc, rout = brute_accept(logits, draft, u, T, k, pnuc)
+    assert np.array_equal(acc, racc) and np.array_equal(out, rout)
+    f = wl.bf16_bits_to_f32(logits).astype(np.float64)
+    for b in range(B):
+        for i in range(gamma + 1):
+            rid, rp = filtered_distribution(f[b, i], T, k, pnuc)
+            assert ids[b, i, :len(rid)].tolist() == rid and (ids[b, i, len(rid):] == -1).all()
+            assert np.abs(pp[b, i, :len(rid)] - rp).max() <= 1e-14
+            assert abs(pp[b, i].sum() - 1.0) <= 1e-14
+
+
+def test_closed_form_two_to_one_distribution():
+    # logits (1, 0, 0) with temperature 1/ln 2  ->  p = (1/2, 1/4, 1/4)
+    T = 1.0 / math.log(2.0)
+    logits = _bits(np.array([[[1.0, 0.0, 0.0], [1.0, 0.0, 0.0]]]))         # gamma = 1
+    _, _, ids, pp = oracle.accept_sample(logits, [[0]], np.zeros((1, 2, 2)), temperature=T, top_k=3, top_p=1.0)
+    assert ids[0, 0].tolist() == [0, 1, 2] and np.allclose(pp[0, 0], [0.5, 0.25, 0.25], rtol=0, atol=1e-15)
+
+    def run(draft, ua, us, **kw):
+        u = np.array([[[ua, us], [0.0, us]]])
+        acc, out, _, _ = oracle.accept_sample(logits, [[draft]], u, temperature=T, top_k=3, **kw)
+        return int(acc[0]), out[0].tolist()
+
+    assert run(0, 0.499, 0.9, top_p=1.0) == (1, [0, 2])        # accepted, bonus from (1/2,1/4,1/4) at 0.9 -> token 2
+    assert run(0, 0.501, 0.4, top_p=1.0) == (0, [1, -1])       # rejected: residual (1/2, 1/2) over tokens 1, 2
+    assert run(0, 0.501, 0.6, top_p=1.0) == (0, [2, -1])
+    assert run(1, 0.249, 0.6, top_p=1.0) == (1, [1, 1])        # bonus: cumulative 0.5, 0.75 -> 0.6 picks token 1
+    assert run(1, 0.251, 0.6, top_p=1.0) == (0, [0, -1])       # residual (2/3, 1/3) over tokens 0, 2
+    assert run(1, 0.251, 0.7, top_p=1.0) == (0, [2, -1])
+    # nucleus 0.7: keep tokens 0 and 1 (the tie between 1 and 2 goes to the lower index), renormalised (2/3, 1/3)
+    _, _, ids, pp = oracle.accept_sample(logits, [[0]], np.zeros((1, 2, 2)), temperature=T, top_k=3, top_p=0.7)
+    assert ids[0, 0].tolist() == [0, 1, -1] and np.allclose(pp[0, 0], [2 / 3, 1 / 3, 0], rtol=0, atol=1e-15)
+    assert run(2, 0.0, 0.5, top_p=0.7) == (0, [0, -1])         # a draft outside the nucleus is always rejected
+    assert run(1, 0.33, 0.9, top_p=0.7) == (1, [1, 1])
+
+
+def test_output_distribution_equals_target_distribution():
+    # losslessness: integrate over a fine lattice of (u_accept, u_sample); whatever the draft token,
+    # the emitted token follows p exactly
+    rng = np.random.default_rng(1)
+    V, N = 7, 400
+    x = rng.standard_normal((1, 2, V)).astype(np.float32) * 2
+    logits = _bits(x)
+    T, k, pnuc = 0.7, 5, 0.9
+    ids, p = filtered_distribution(wl.bf16_bits_to_f32(logits)[0, 0].astype(np.float64), T, k, pnuc)
+    grid = (np.arange(N) + 0.5) / N
+    ua, us = np.meshgrid(grid, grid, indexing="ij")
+    u = np.zeros((N * N, 2, 2))
+    u[:, 0, 0], u[:, 0, 1] = ua.ravel(), us.ravel()
+    big = np.broadcast_to(logits, (N * N, 2, V)).copy()
+    for draft_tok in (ids[0], ids[-1], int(np.argmin(x[0, 0]))):
+        acc, out, _, _ = oracle.accept_sample(big, np.full((N * N, 1), draft_tok), u, temperature=T, top_k=k, top_p=pnuc)
+        freq = np.bincount(out[:, 0], minlength=V) / (N * N)
+        want = np.zeros(V)
+        want[ids] = p
+        assert np.abs(freq - want).max() <= 2.5 / N
+
+
+def test_top_k_one_or_tiny_nucleus_is_greedy():
+    B, gamma, V = 6, 5, 3000
+    logits = wl.make_logits(B, gamma, V, seed=9)
+    best, _, _ = oracle.accept_greedy(logits, np.zeros((B, gamma), np.int32))
+    draft, cut = wl.make_draft(best, V, seed=9)
+    gt, ga, go = oracle.accept_greedy(logits, draft)
+    u = np.random.default_rng(0).random((B, gamma + 1, 2))
+    for kw in (dict(temperature=0.7, top_k=1, top_p=0.8), dict(temperature=1.3, top_k=20, top_p=1e-9),
+               dict(temperature=1e-3, top_k=20, top_p=0.999)):
+        acc, out, _, _ = oracle.accept_sample(logits, draft, u, **kw)
+        assert np.array_equal(acc, ga) and np.array_equal(out, go)
+
+
+def test_nan_never_a_candidate_and_masked_vocabulary():
+    x = np.full((1, 1, 10), -np.inf, np.float32)
+    x[0, 0, 3] = np.nan
+    x[0, 0, 7] = 1.0
+    x[0, 0, 8] = 1.0
+    acc, out, ids, pp = oracle.accept_sample(_bits(x), np.zeros((1, 0), np.int32), np.array([[[0.0, 0.75]]]),
+                                             temperature=1.0, top_k=4, top_p=1.0)
+    assert ids[0, 0, :2].tolist() == [7, 8] and 3 not in ids[0, 0]
+    assert np.allclose(pp[0, 0, :2], [0.5, 0.5]) and np.allclose(pp[0, 0, 2:], 0)
+    assert out[0, 0] == 8 and acc[0] == 0
