@@ -199,6 +199,26 @@ class Accept:
                                   self.tok, self.ws)
 
 
+class Sample:
+    """ts_accept_sample on the same logits / drafts as an Accept instance (paper's sampling regime)."""
+
+    def __init__(self, acc: "Accept", seed=0, temperature=0.7, top_k=20, top_p=0.8):
+        import torch
+        self.api, self.acc = acc.api, acc
+        self.kw = dict(temperature=temperature, top_k=top_k, top_p=top_p)
+        rng = np.random.default_rng([seed, 17])
+        self.u = torch.from_numpy(rng.random((acc.B, acc.gamma + 1, 2), dtype=np.float32)).cuda()
+        self.alen = torch.empty((acc.B,), dtype=torch.int32, device="cuda")
+        self.tok = torch.empty((acc.B, acc.gamma + 1), dtype=torch.int32, device="cuda")
+        self.ws = torch.empty(acc.api.sample_workspace_bytes(acc.B, acc.gamma, acc.V, top_k), dtype=torch.uint8,
+                              device="cuda")
+
+    def run(self):
+        a = self.acc
+        self.api.ts_accept_sample(a.logits, a.draft if a.gamma > 0 else None, self.u, self.alen, self.tok, self.ws,
+                                  **self.kw)
+
+
 class L2Flusher:
     def __init__(self, nbytes=512 << 20):
         import torch
@@ -517,7 +537,13 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         record(f"verify_g{g}:ts_accept_greedy", acc.bytes, amed, amn, emitted,
                {"emitted_tokens": emitted, "accepted_equals_seeded_cuts": bool((acc.acc.cpu().numpy() == acc.cut).all())})
         out[f"verify_g{g}:emitted_tokens_per_s"] = emitted / ((med + amed) * 1e-3)
-        del acc
+        smp = Sample(acc, seed=seed)
+        smed, smn = time_with_flush(smp.run, flush)
+        semitted = int((smp.alen + 1).sum().item())
+        record(f"verify_g{g}:ts_accept_sample", acc.bytes, smed, smn, semitted,
+               {"emitted_tokens": semitted, "temperature": 0.7, "top_k": 20, "top_p": 0.8,
+                "note": "drafts = row argmax up to the seeded cut point; acceptance is stochastic here"})
+        del acc, smp
 
     # concurrency sweep on the mixed length pool: attention-only analogue of v(b) and b*v(b)
     pool_lens = wl.lens_mixed(seed)
@@ -567,13 +593,14 @@ def run_profile_case(args):
         lens, ql = wl.lens_tail(0)[:2], 1
     elif name.startswith("verify4_g"):
         lens, ql = wl.lens_verify(0)[:4], 1 + int(name[len("verify4_g"):])
-    elif name.startswith("accept_g"):
+    elif name.startswith("accept_g") or name.startswith("sample_g"):
         g = int(name[len("accept_g"):])
         acc = Accept(16, g, seed=0)
+        obj = Sample(acc, seed=0) if name.startswith("sample_g") else acc
         flush = L2Flusher(256 << 20)
         for _ in range(3):
             flush()
-            acc.run()
+            obj.run()
         torch.cuda.synchronize()
         print(json.dumps({"profile_case": name, "bytes": acc.bytes}))
         return 0
@@ -602,7 +629,7 @@ def main():
     ap.add_argument("--ncu-traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the attention kernel from an ncu capture (reported as roofline.traffic)")
     ap.add_argument("--profile-case", default=None,
-                    help="run a small case for a profiler capture: bulk64, tail2, verify4_g4|8|16, accept_g4|8|16")
+                    help="run a small case for a profiler capture: bulk64, tail2, verify4_g4|8|16, accept_g4|8|16, sample_g4|8|16")
     args = ap.parse_args()
     if args.profile_case:
         return run_profile_case(args)

@@ -160,6 +160,37 @@ int ts_accept_greedy(const void *logits, int64_t row_stride, const int32_t *draf
                      int32_t gamma, int32_t vocab, int32_t *target_argmax, int32_t *accept_len,
                      int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Scratch bytes for ts_accept_sample (host-only; 0 for sizes it does not support). */
+size_t ts_sample_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab, int32_t top_k);
+
+/*
+ * Lossless acceptance of a draft block under the paper's rollout sampling regime -- temperature,
+ * top-k and top-p (Appendix, Table "shared-sampling-config": 0.7 / 20 / 0.8) -- with the speculative
+ * sampling rule of Section 3.4, for drafters that propose one token per position (point proposals,
+ * draft distribution = one-hot).  Per logits row: the top_k largest logits (equal logits ordered by
+ * ascending index, NaN never selected); p = softmax(logit / temperature) over them; the shortest
+ * prefix whose probability reaches top_p is kept and renormalised.  Per sequence, with the uniforms
+ * u[b, i, 0] (accept) and u[b, i, 1] (sample), i = 0 .. gamma, all in [0, 1):
+ *   the draft token x_i is accepted iff it is kept and u_accept < p(x_i); at the first rejection
+ *   one token is drawn from p with x_i removed (inverse CDF over the kept order, renormalised) and
+ *   the walk stops; if all gamma drafts are accepted one more token is drawn from p_gamma.
+ * The emitted tokens follow the target distribution exactly, whatever the drafts.
+ *   logits      bf16, row (b, i) at logits + (b*(gamma+1)+i)*row_stride; row_stride and vocab
+ *               multiples of 8 (16-byte aligned rows)
+ *   draft       int32 [num_seqs, gamma] (may be NULL when gamma == 0)
+ *   uniforms    fp32 [num_seqs, gamma+1, 2]
+ *   accept_len  int32 [num_seqs]; out_tokens int32 [num_seqs, gamma+1], -1 padded
+ *   workspace   >= ts_sample_workspace_bytes(...) bytes, clobbered
+ * temperature > 0, 1 <= top_k <= 32, 0 < top_p <= 1, vocab <= 524288.  Token selection is exact;
+ * probabilities are fp32, so a uniform within rounding of a probability may decide either way.
+ * Penalties on already generated tokens (the paper's presence penalty) are the caller's job: apply
+ * them to the logits first.
+ */
+int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draft, const float *uniforms,
+                     int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k,
+                     float top_p, int32_t *accept_len, int32_t *out_tokens, void *workspace,
+                     size_t workspace_bytes, void *stream);
+
 /*
  * ts_accept_greedy for callers that have no device memory to give and cannot get any.  (The paper
  * has no counterpart; this is a packaging variant of ts_accept_greedy.)  Who that is: a serving

@@ -22,7 +22,7 @@ TS_OK = 0
 EXPORTED_SYMBOLS = (
     "ts_attn_workspace_bytes", "ts_splitkv_workspace_bytes", "ts_decode_attn", "ts_verify_attn",
     "ts_decode_attn_splitkv", "ts_lse_merge", "ts_accept_workspace_bytes", "ts_accept_greedy",
-    "ts_accept_greedy_noalloc",
+    "ts_accept_greedy_noalloc", "ts_sample_workspace_bytes", "ts_accept_sample",
     "ts_set_attn_timing_events", "ts_status_string",
 )
 
@@ -73,6 +73,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ts_accept_greedy.argtypes = [vp, i64, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     lib.ts_accept_greedy_noalloc.restype = ctypes.c_int
     lib.ts_accept_greedy_noalloc.argtypes = [vp, i64, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.ts_sample_workspace_bytes.restype = sz
+    lib.ts_sample_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    lib.ts_accept_sample.restype = ctypes.c_int
+    lib.ts_accept_sample.argtypes = [vp, i64, vp, vp, i32, i32, i32, ctypes.c_float, i32, ctypes.c_float, vp, vp, vp, sz, vp]
     lib.ts_set_attn_timing_events.restype = ctypes.c_int
     lib.ts_set_attn_timing_events.argtypes = [vp, vp]
     lib.ts_status_string.restype = ctypes.c_char_p
@@ -229,3 +233,22 @@ def ts_accept_greedy_noalloc(logits, draft, target_argmax, accept_len, out_token
                                       _ptr(accept_len, "accept_len"), _ptr(out_tokens, "out_tokens"), _stream())
     _check(rc, "ts_accept_greedy_noalloc")
     return target_argmax, accept_len, out_tokens
+
+
+def sample_workspace_bytes(num_seqs: int, gamma: int, vocab: int, top_k: int) -> int:
+    return int(load_library().ts_sample_workspace_bytes(num_seqs, gamma, vocab, top_k))
+
+
+def ts_accept_sample(logits, draft, uniforms, accept_len, out_tokens, workspace, *, temperature: float, top_k: int,
+                     top_p: float, row_stride=None):
+    """Lossless draft acceptance under temperature / top-k / top-p sampling (see the header)."""
+    lib = load_library()
+    B, R, V = logits.shape
+    gamma = R - 1
+    stride = int(row_stride) if row_stride is not None else int(logits.stride(1))
+    rc = lib.ts_accept_sample(_ptr(logits, "logits"), stride, _ptr(draft, "draft") if gamma > 0 else None,
+                              _ptr(uniforms, "uniforms"), B, gamma, V, float(temperature), int(top_k), float(top_p),
+                              _ptr(accept_len, "accept_len"), _ptr(out_tokens, "out_tokens"),
+                              _ptr(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "ts_accept_sample")
+    return accept_len, out_tokens

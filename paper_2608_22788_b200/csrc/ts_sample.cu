@@ -1,0 +1,370 @@
+// Lossless draft acceptance under temperature / top-k / top-p sampling for sm_100a.
+//
+// Kernel 1 streams the logits once (HBM-bound, same register-resident chunks as the greedy argmax)
+// and leaves the top_k best (value, index) pairs of every chunk; kernel 2 (one CTA per sequence)
+// merges the chunks of each row, builds the filtered distribution and walks the draft block.
+// Selection is exact and integer-only (ordered bf16 keys, ties to the lower index); probabilities
+// are fp32.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#include "../../include/tailsieve.h"
+#include "ts_common.cuh"
+
+namespace ts {
+namespace smp {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerThread = 16;
+constexpr int kChunkMax = kThreads * kVecPerThread * 8;      // 32768 logits per chunk
+constexpr int kMaxTopK = 32;
+constexpr int kMaxChunks = 16;
+constexpr int kCap = 2048;                                   // candidate slots per chunk
+
+__device__ __forceinline__ uint32_t bf16_key(uint32_t u)
+{
+    u &= 0xffffu;
+    if ((u & 0x7fffu) > 0x7f80u) return 0u;          // NaN: below everything
+    if (u == 0x8000u) u = 0u;                          // -0 -> +0
+    const uint32_t ord = (u & 0x8000u) ? (~u & 0xffffu) : (u | 0x8000u);
+    return ord + 1u;
+}
+// Inverse of bf16_key for keys >= 1 (returns +0 for the zero key).
+__device__ __forceinline__ uint32_t key_to_bf16(uint32_t key)
+{
+    const uint32_t ord = key - 1u;
+    return (ord & 0x8000u) ? (ord & 0x7fffu) : (~ord & 0xffffu);
+}
+__device__ __forceinline__ uint4 ld_stream_16B(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned long long pack_key(uint32_t key16, int idx)
+{
+    return ((unsigned long long)key16 << 32) | (unsigned long long)(0xffffffffu - (uint32_t)idx);
+}
+
+__device__ __noinline__ void push_candidates(uint4 v, uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, int idx0,
+                                             int *cnt, unsigned long long *cand)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const uint32_t e[4] = {e0, e1, e2, e3};
+    for (int i = 0; i < 4; ++i) {
+        if (e[i] & 0xffffu) { const int s = atomicAdd(cnt, 1); if (s < kCap) cand[s] = pack_key(bf16_key(w[i]), idx0 + 2 * i); }
+        if (e[i] >> 16) { const int s = atomicAdd(cnt, 1); if (s < kCap) cand[s] = pack_key(bf16_key(w[i] >> 16), idx0 + 2 * i + 1); }
+    }
+}
+
+// Degenerate chunk (thousands of ties at the threshold): extract the best key below the previous
+// one, top_k times, re-reading the chunk from memory each time.  Slow, exact, and only reached by
+// pathological inputs such as a constant row.
+__device__ __noinline__ void slow_topk(const uint4 *base, int nvec, int begin, int top_k, unsigned long long *dst,
+                                       unsigned long long *s_red)
+{
+    const int tid = threadIdx.x;
+    unsigned long long prev = ~0ull;
+    for (int r = 0; r < top_k; ++r) {
+        unsigned long long best = 0ull;
+        for (int j = tid; j < nvec; j += kThreads) {
+            const uint4 x = base[j];
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+            const int idx0 = begin + j * 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t ka = bf16_key(w[i]), kb = bf16_key(w[i] >> 16);
+                const unsigned long long a = pack_key(ka, idx0 + 2 * i), b = pack_key(kb, idx0 + 2 * i + 1);
+                if (ka && a < prev && a > best) best = a;
+                if (kb && b < prev && b > best) best = b;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { const unsigned long long x = __shfl_xor_sync(0xffffffffu, best, o); best = x > best ? x : best; }
+        if ((tid & 31) == 0) s_red[tid >> 5] = best;
+        __syncthreads();
+        best = s_red[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) best = s_red[w] > best ? s_red[w] : best;
+        __syncthreads();
+        if (tid == 0) dst[r] = best;
+        if (best == 0ull) break;
+        prev = best;
+    }
+}
+
+// grid = (chunks, rows).  out[(row * chunks + chunk) * top_k + j] = j-th best key of the chunk (0 = none).
+__global__ void __launch_bounds__(kThreads, 3)
+ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len, int top_k,
+                     unsigned long long *__restrict__ out)
+{
+    __shared__ unsigned long long s_cand[kCap];
+    __shared__ unsigned long long s_red[kThreads / 32];
+    __shared__ int s_cnt;
+    __shared__ uint32_t s_tkey[kThreads];
+    __shared__ uint32_t s_t1;
+    const int chunk = blockIdx.x, row = blockIdx.y, chunks = gridDim.x;
+    const int tid = threadIdx.x;
+    const int begin = chunk * chunk_len;
+    int end = begin + chunk_len;
+    if (end > vocab) end = vocab;
+    const int nvec = end > begin ? (end - begin) >> 3 : 0;
+    const uint4 *base = reinterpret_cast<const uint4 *>(logits + (long long)row * row_stride + begin);
+    unsigned long long *dst = out + ((long long)row * chunks + chunk) * top_k;
+    const uint32_t nan2 = 0x7fc07fc0u;
+    uint4 v[kVecPerThread];
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+        const int j = tid + u * kThreads;
+        v[u] = j < nvec ? ld_stream_16B(base + j) : make_uint4(nan2, nan2, nan2, nan2);
+    }
+    if (tid == 0) s_cnt = 0;
+    // ---- the largest element of every thread (NaN never wins)
+    __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162 *>(&nan2);
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&v[u].x));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&v[u].y));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&v[u].z));
+        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&v[u].w));
+    }
+    const uint32_t mbits = *reinterpret_cast<const uint32_t *>(&m2);
+    const uint32_t k0 = bf16_key(mbits), k1 = bf16_key(mbits >> 16);
+    const uint32_t tkey = k0 > k1 ? k0 : k1;
+    // ---- threshold T1 = the top_k-th largest of the 256 thread maxima (0 if fewer than top_k threads
+    //      hold a number): the top_k-th largest element of the chunk is >= T1, so the chunk's top_k are
+    //      all >= T1, and on random data only a few dozen elements are.  Warp 0 finds it by binary search
+    //      on the 17-bit key, counting with ballots over the 8 maxima each of its lanes holds.
+    s_tkey[tid] = tkey;
+    __syncthreads();
+    if (tid < 32) {
+        uint32_t k8[kThreads / 32];
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) k8[i] = s_tkey[tid + 32 * i];
+        const int want = top_k < kThreads ? top_k : kThreads;
+        uint32_t lo = 0u, hi = 65537u;                    // count(>= lo) >= want holds for lo = 0
+        while (hi - lo > 1u) {
+            const uint32_t mid = (lo + hi) >> 1;
+            int c = 0;
+#pragma unroll
+            for (int i = 0; i < kThreads / 32; ++i) c += __popc(__ballot_sync(0xffffffffu, k8[i] >= mid));
+            if (c >= want) lo = mid; else hi = mid;
+        }
+        if (tid == 0) s_t1 = lo;
+    }
+    __syncthreads();
+    const uint32_t t1 = s_t1;
+    const uint32_t t1bits = t1 ? key_to_bf16(t1) : 0xff80u;          // no k-th maximum: everything that is not NaN
+    const uint32_t t1x2 = t1bits | (t1bits << 16);
+    const __nv_bfloat162 tt = *reinterpret_cast<const __nv_bfloat162 *>(&t1x2);
+    // ---- candidates (rare: a few hundred of the chunk's 32768 elements; the push is kept out of line
+    //      so that the unrolled scan stays small)
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+        const uint32_t e0 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].x), tt);
+        const uint32_t e1 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].y), tt);
+        const uint32_t e2 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].z), tt);
+        const uint32_t e3 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].w), tt);
+        if (e0 | e1 | e2 | e3) push_candidates(v[u], e0, e1, e2, e3, begin + (tid + u * kThreads) * 8, &s_cnt, s_cand);
+    }
+    for (int j = tid; j < top_k; j += kThreads) dst[j] = 0ull;
+    __syncthreads();
+    const int cnt = s_cnt;
+    if (cnt <= kCap) {
+        // ---- rank the candidates; the best top_k go out in order
+        for (int c = tid; c < cnt; c += kThreads) {
+            const unsigned long long mine = s_cand[c];
+            int rank = 0;
+            for (int j = 0; j < cnt; ++j) rank += s_cand[j] > mine;
+            if (rank < top_k) dst[rank] = mine;
+        }
+    } else {
+        slow_topk(base, nvec, begin, top_k, dst, s_red);
+    }
+}
+
+// One CTA per sequence, one warp per row (rows beyond the number of warps are taken in turn); warp 0
+// then walks the draft block with one kept token per lane.
+__global__ void __launch_bounds__(1024)
+ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks, int top_k,
+                        const uint16_t *__restrict__ logits, long long row_stride, const int32_t *__restrict__ draft,
+                        const float *__restrict__ uniforms, int gamma, float inv_temperature, float top_p,
+                        int32_t *accept_len, int32_t *out_tokens)
+{
+    extern __shared__ unsigned char smem[];
+    constexpr uint32_t FULL = 0xffffffffu;
+    const int R = gamma + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int total = chunks * top_k;
+    int32_t *s_ids = reinterpret_cast<int32_t *>(smem);                       // [R][32]
+    float *s_p = reinterpret_cast<float *>(smem + (size_t)R * 32 * 4);         // [R][32]
+    unsigned long long *s_best = reinterpret_cast<unsigned long long *>(smem + (size_t)R * 32 * 8);   // [warps][32]
+    unsigned long long *s_cand = s_best + nwarps * 32;                         // [warps][chunks * top_k]
+    grid_dependency_wait();       // the chunk keys of the kernel before
+    const int b = blockIdx.x;
+    for (int i = warp; i < R; i += nwarps) {
+        const long long row = (long long)b * R + i;
+        const unsigned long long *src = keys + row * total;
+        unsigned long long *best = s_best + warp * 32;
+        unsigned long long *cand = s_cand + (size_t)warp * total;
+        best[lane] = 0ull;
+        for (int c = lane; c < total; c += 32) cand[c] = src[c];
+        __syncwarp();
+        for (int c = lane; c < total; c += 32) {
+            const unsigned long long mine = cand[c];
+            if (mine == 0ull) continue;
+            int rank = 0;
+            for (int j = 0; j < total; ++j) rank += cand[j] > mine;
+            if (rank < top_k) best[rank] = mine;
+        }
+        __syncwarp();
+        const unsigned long long key = best[lane];
+        const bool valid = lane < top_k && key != 0ull;
+        const int idx = valid ? (int)(0xffffffffu - (uint32_t)(key & 0xffffffffull)) : -1;
+        // the logit itself (bf16 -> fp32, exact)
+        float x = -INFINITY;
+        if (valid) x = __uint_as_float((uint32_t)logits[row * row_stride + idx] << 16);
+        const float z = x * inv_temperature;
+        const float z0 = __shfl_sync(FULL, z, 0);
+        float e = valid ? expf(z - z0) : 0.f;
+        if (valid && z == z0) e = 1.f;                                           // also covers z0 = -inf
+        float sum = e;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+        const float p = sum > 0.f ? e / sum : 0.f;
+        float cum = p;                                                            // inclusive prefix sum in rank order
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const float y = __shfl_up_sync(FULL, cum, o); if (lane >= o) cum += y; }
+        const bool keep = valid && (lane == 0 || (cum - p) < top_p);
+        // nucleus membership must be a prefix: a lane is kept only if every earlier one is
+        const unsigned kept_mask = __ballot_sync(FULL, keep);
+        const int nkept = kept_mask == FULL ? 32 : __ffs(~kept_mask) - 1;          // length of the leading run of ones
+        const bool kept = lane < nkept;
+        float ks = kept ? p : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ks += __shfl_xor_sync(FULL, ks, o);
+        s_ids[i * 32 + lane] = kept ? idx : -1;
+        s_p[i * 32 + lane] = kept ? p / ks : 0.f;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int32_t *out = out_tokens + (long long)b * R;
+        for (int i = lane; i < R; i += 32) out[i] = -1;
+        __syncwarp();
+        int a = 0;
+        for (int i = 0; i <= gamma; ++i) {
+            const int32_t id = s_ids[i * 32 + lane];
+            const float pj = s_p[i * 32 + lane];
+            const float ua = uniforms[((long long)b * R + i) * 2], us = uniforms[((long long)b * R + i) * 2 + 1];
+            bool is_draft = false;
+            if (i < gamma) {
+                const int32_t xtok = draft[(long long)b * gamma + i];
+                is_draft = (id == xtok) && id >= 0;
+                const unsigned hit = __ballot_sync(FULL, is_draft);
+                const float px = hit ? __shfl_sync(FULL, pj, __ffs(hit) - 1) : 0.f;
+                if (ua < px) {                      // accepted: next position
+                    if (lane == 0) out[i] = xtok;
+                    ++a;
+                    continue;
+                }
+            }
+            // one token from the (residual) distribution, then stop
+            const float w = (id >= 0 && !is_draft) ? pj : 0.f;
+            float cum = w, tot = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const float y = __shfl_up_sync(FULL, cum, o); if (lane >= o) cum += y; }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(FULL, tot, o);
+            const bool live = id >= 0 && !is_draft;
+            const unsigned over = __ballot_sync(FULL, live && cum > us * tot);
+            const unsigned lives = __ballot_sync(FULL, live);
+            int pick = -1;
+            if (over) pick = __ffs(over) - 1;
+            else if (lives) pick = 31 - __clz(lives);          // rounding left the last one
+            const int32_t y = pick >= 0 ? __shfl_sync(FULL, id, pick) : -1;
+            if (lane == 0) out[i] = y;
+            break;
+        }
+        if (lane == 0) accept_len[b] = a;
+    }
+}
+
+static int pick_chunks(long long rows, int vocab)
+{
+    // a chunk must fit in registers; beyond that, only as many chunks as it takes to have about two
+    // CTAs per SM (every CTA pays a fixed selection overhead)
+    const int need = (vocab + kChunkMax - 1) / kChunkMax;
+    long long c = (296 + rows - 1) / rows;
+    const long long by_len = (vocab + 4095) / 4096;
+    if (c > by_len) c = by_len;
+    if (c > kMaxChunks) c = kMaxChunks;
+    if (c < need) c = need;
+    return (int)c;
+}
+
+}  // namespace smp
+}  // namespace ts
+
+extern "C" {
+
+size_t ts_sample_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab, int32_t top_k)
+{
+    if (num_seqs < 0 || gamma < 0 || vocab < 1 || top_k < 1 || top_k > ts::smp::kMaxTopK) return 0;
+    if ((vocab + ts::smp::kChunkMax - 1) / ts::smp::kChunkMax > ts::smp::kMaxChunks) return 0;
+    const size_t bytes = (size_t)num_seqs * (gamma + 1) * ts::smp::kMaxChunks * top_k * sizeof(unsigned long long);
+    return bytes < 256 ? 256 : bytes;
+}
+
+int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draft, const float *uniforms,
+                     int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k, float top_p,
+                     int32_t *accept_len, int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace ts::smp;
+    if (num_seqs < 0 || gamma < 0 || vocab < 1) return TS_ERR_INVALID_ARG;
+    if (!logits || !uniforms || !accept_len || !out_tokens || !workspace) return TS_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft) return TS_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || isinf(temperature) || !(top_p > 0.f) || top_p > 1.f) return TS_ERR_INVALID_ARG;
+    if (top_k < 1) return TS_ERR_INVALID_ARG;
+    if (top_k > kMaxTopK || gamma > 255) return TS_ERR_UNSUPPORTED;
+    if (row_stride < vocab) return TS_ERR_INVALID_ARG;
+    if (row_stride % 8 != 0 || vocab % 8 != 0) return TS_ERR_UNSUPPORTED;      // rows must be 16-byte aligned
+    if ((vocab + kChunkMax - 1) / kChunkMax > kMaxChunks) return TS_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(logits) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return TS_ERR_INVALID_ARG;
+    const size_t need = ts_sample_workspace_bytes(num_seqs, gamma, vocab, top_k);
+    if (need == 0) return TS_ERR_UNSUPPORTED;
+    if (workspace_bytes < need) return TS_ERR_WORKSPACE;
+    const long long rows = (long long)num_seqs * (gamma + 1);
+    if (rows == 0) return TS_OK;
+    if (rows > 65535) return TS_ERR_UNSUPPORTED;
+    const int chunks = pick_chunks(rows, vocab);
+    int chunk_len = (vocab + chunks - 1) / chunks;
+    chunk_len = (chunk_len + 7) / 8 * 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned long long *keys = static_cast<unsigned long long *>(workspace);
+    ts_topk_chunk_kernel<<<dim3((unsigned)chunks, (unsigned)rows), kThreads, 0, s>>>(
+        static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, top_k, keys);
+    if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+    const int R = gamma + 1;
+    int warps = R < 32 ? R : 32;
+    size_t smem;
+    for (;;) {
+        smem = (size_t)R * 32 * 8 + (size_t)warps * 32 * 8 + (size_t)warps * chunks * top_k * 8;
+        if (smem <= 48 * 1024 || warps == 1) break;
+        warps = (warps + 1) / 2;
+    }
+    if (smem > 48 * 1024) return TS_ERR_UNSUPPORTED;
+    const char *pdl = getenv("TS_PDL");
+    const bool overlap = !(pdl && pdl[0] == '0');
+    const cudaError_t e = ts::launch_overlapped(ts_sample_finish_kernel, dim3((unsigned)num_seqs), dim3(warps * 32), smem, s,
+                                                overlap, (const unsigned long long *)keys, chunks, (int)top_k,
+                                                static_cast<const uint16_t *>(logits), (long long)row_stride, draft,
+                                                uniforms, (int)gamma, 1.0f / temperature, top_p, accept_len, out_tokens);
+    return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
+}
+
+}  // extern "C"
