@@ -139,6 +139,19 @@ int ts_decode_attn_splitkv(const ts_attn_params *p, const void *q, const void *k
 int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *partial_o,
                  const float *partial_lse, const int32_t *num_splits, void *out, void *stream);
 
+/*
+ * Writes the K and V rows of the q_len tokens scored in this step into the paged cache, so that the
+ * attention calls above find them there (the step before attention; the paper's decode step appends
+ * one token per request, its verify step 1 + gamma -- Sections 2.1 and 3.4).
+ *   new_k, new_v  bf16 [num_seqs, q_len, num_kv_heads, head_dim], contiguous
+ *   Token t of sequence s goes to position kv_lens[s] - q_len + t (kv_lens already counts the new
+ *   tokens, as in the attention calls), i.e. page block_table[s, pos / page_size], slot
+ *   pos % page_size.  Positions below 0 are skipped.  Bit-exact copy; needs head_dim % 8 == 0.
+ *   Uses q_len, num_kv_heads, head_dim, page_size, max_pages_per_seq and the three strides of `p`.
+ */
+int ts_kv_append(const ts_attn_params *p, const void *new_k, const void *new_v, void *k_pool, void *v_pool,
+                 const int32_t *block_table, const int32_t *kv_lens, void *stream);
+
 /* Scratch bytes for ts_accept_greedy (host-only; 0 for invalid sizes). */
 size_t ts_accept_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab);
 

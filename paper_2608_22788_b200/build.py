@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libtailsieve.so")
-SOURCES = ["ts_attn.cu", "ts_accept.cu", "ts_sample.cu"]
+SOURCES = ["ts_attn.cu", "ts_accept.cu", "ts_sample.cu", "ts_append.cu"]
 HEADERS = [os.path.join(CSRC, "ts_common.cuh"), os.path.join(CSRC, "ts_attn_tc.cuh"),
            os.path.join(os.path.dirname(_HERE), "include", "tailsieve.h")]
 
