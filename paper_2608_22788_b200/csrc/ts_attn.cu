@@ -610,35 +610,39 @@ __device__ __forceinline__ void merge_row(const float *po, size_t o_stride, cons
     }
 }
 
-// Free mode: one CTA (4 warps, one output row each at a time) per (s, g) pair; pairs covered by a
-// single group are skipped.
+// Free mode: one CTA per group of the tile line.  CTA k merges the pair that straddles the end of
+// group k's piece if that pair starts inside the piece (so every split pair is merged exactly once,
+// by the group that holds its first part), and zero-fills the outputs of empty sequences k, k+NG, ...
+// Pairs covered by a single group were written directly by the attention kernel.
 template <int D>
 __global__ void __launch_bounds__(128)
-ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const float *__restrict__ part_o,
+ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__restrict__ gstart,
+                     const long long *__restrict__ gpos, const float *__restrict__ part_o,
                      const float *__restrict__ part_lse, uint16_t *out, int B, int q_len, int Hq, int Hkv,
                      int NG)
 {
     grid_dependency_wait();       // partials and direct outputs of the attention kernel
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = blockIdx.x;
-    const int s = pair / Hkv, g = pair % Hkv;
+    const int k_first = blockIdx.x;
     const int G = Hq / Hkv, rows = G * q_len;
+    // ---- empty sequences: zeros
+    for (int s0 = k_first; s0 < B; s0 += NG) {
+        if (cum_tiles[s0 + 1] != cum_tiles[s0]) continue;
+        uint32_t *o = reinterpret_cast<uint32_t *>(out + (size_t)s0 * q_len * Hq * D);
+        for (int i = threadIdx.x; i < q_len * Hq * D / 2; i += 128) o[i] = 0u;
+    }
+    // ---- the pair cut by the end of this group's piece
+    const GroupStart nx = gstart[k_first + 1];
+    if (nx.s >= B || nx.tau == 0) return;                  // the piece ends on a pair boundary
+    const int s = nx.s, g = nx.g;
     const int tiles = cum_tiles[s + 1] - cum_tiles[s];
     const long long W = (long long)Hkv * cum_tiles[B];
-    int k_first = 0, k_last = -1;
-    if (tiles > 0) {
-        const long long a0 = (long long)Hkv * cum_tiles[s] + (long long)g * tiles, b0 = a0 + tiles;
-        k_first = (int)(((a0 + 1) * NG - 1) / W);
-        k_last = (int)((b0 * NG - 1) / W);
-        if (k_first == k_last) return;      // written directly by the attention kernel
-    }
+    const long long a0 = gpos[k_first + 1] - nx.tau, b0 = a0 + tiles;
+    if (a0 < gpos[k_first]) return;                        // the pair started in an earlier group: merged there
+    const int k_last = (int)((b0 * NG - 1) / W);
     for (int r = warp; r < rows; r += 4) {
         const int t = r / G, hl = r % G;
         uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
-        if (tiles == 0) {
-            merge_row<D>(nullptr, 0, nullptr, 0, 0, orow, lane);
-            continue;
-        }
         // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
         // (pair started before them).
         // Groups whose piece of the tile line is empty (only when W < NG) wrote nothing: skip them.
@@ -1040,15 +1044,16 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
 
     if (free_mode) {
         const bool overlap = env_int("TS_PDL", 1) != 0;
-        const int pairs = a.B * a.Hkv;
-        const dim3 mgrid((unsigned)pairs);
+        const dim3 mgrid((unsigned)NG);
         cudaError_t e;
         if (p->head_dim == 128)
-            e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles,
-                                  (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq, a.Hkv, NG);
+            e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles, a.gstart,
+                                  a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
+                                  a.Hkv, NG);
         else
-            e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles,
-                                  (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq, a.Hkv, NG);
+            e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles, a.gstart,
+                                  a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
+                                  a.Hkv, NG);
         if (e != cudaSuccess) return TS_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
     }
