@@ -586,6 +586,19 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
                          "kv_tokens": [r[3] for r in rows], "draws": draws}
     out["concurrency_sweep:ts_decode_attn"] = sweep
 
+    # the paper's all-admit completion-time model (Section 2.1, Appendix D) fed with the measured
+    # attention-only tau(b): 1024 requests whose remaining lengths follow the mixed pool, 8 replicas,
+    # uniform round robin versus top-k tail isolation with 2 of the 8 replicas as the tail pool
+    from paper_2608_22788_b200 import makespan as mk
+    tau = mk.tau_from_samples([int(c) for c in sweep], [sweep[c]["ms_median"] * 1e-3 for c in sweep])
+    remaining = (pool_lens // 8).tolist()                   # keep the exact per-position sums cheap
+    k_best, t_best, t_uniform = mk.best_topk(remaining, tau, tail_replicas=2, bulk_replicas=6,
+                                             ks=[1, 2, 4, 8, 16, 32, 64, 128, 256])
+    out["makespan_model"] = {"replicas": 8, "tail_replicas": 2, "requests": len(remaining),
+                             "uniform_s": t_uniform, "best_topk_s": t_best, "best_k": k_best,
+                             "speedup": t_uniform / t_best if t_best > 0 else None,
+                             "note": "tau(b) is the measured attention-only step time; the paper's curve is for a whole model"}
+
     # the mixed batch as one uniform call versus a bulk call plus a tail call (lengths >= 16k to the tail)
     lens = pool_lens
     wb = Workload("mixed_bulk", lens[lens < 16384], pool, seed=seed + 7)

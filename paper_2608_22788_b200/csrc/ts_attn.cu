@@ -912,11 +912,13 @@ static int launch_attn(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a
     a.ngrp = ngrp;
     a.ns = ns;
     if (dry) return TS_OK;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};      // per device: the attribute belongs to the device's copy of the kernel
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TS_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(ts_attn_kernel<D, NT, WG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess)
             return TS_ERR_CUDA;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const cudaError_t e = launch_overlapped(ts_attn_kernel<D, NT, WG>, dim3(grid), dim3(ngrp * WG * 32), smem, stream,
                                             env_int("TS_PDL", 1) != 0, tk, tv, a);
@@ -936,11 +938,13 @@ static int launch_attn_tc(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs
     a.ngrp = 1;
     a.ns = tc::kStages;
     if (dry) return TS_OK;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};      // per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TS_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(tc::ts_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess)
             return TS_ERR_CUDA;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const cudaError_t e = launch_overlapped(tc::ts_attn_tc_kernel, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, stream,
                                             env_int("TS_PDL", 1) != 0, tk, tv, a);
