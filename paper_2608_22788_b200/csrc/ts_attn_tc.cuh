@@ -1,6 +1,6 @@
 // Verify-attention kernel on the 5th-generation tensor cores (tcgen05 + TMEM), head_dim 128.
 //
-// Used when the (GQA group x q_len) tile of a (sequence, kv head) pair has more than 8 rows, i.e. for
+// Used when the (GQA group x q_len) tile of a (sequence, kv head) pair has more than 16 rows, i.e. for
 // speculative verification.  The warp-level MMA path tops out at ~550 TFLOP/s on this GPU, which
 // is less than a 68-row tile needs to keep up with HBM; tcgen05.mma has about three times that.
 //
