@@ -54,6 +54,9 @@ struct AttnArgs {
     int B, q_len, Hq, Hkv, G, rows, P, max_pages, max_splits, mode;
     int ngrp, ns;                // groups per CTA, pipeline stages per group
     int tok_first;               // 1: token is tensor-map dim 1 and head dim 2; 0: the reverse
+    int box_tok;                 // warp-MMA kernel: tokens per 4-D TMA box (16/32/64, <= page size); 0 = one 5-D box per tile
+    int lg_page;                 // log2(page size)
+    int lg_box;                  // log2(box_tok) when box_tok > 0
     float scale_log2;            // scale * log2(e)
     long long wait_cycles;       // bound of every mbarrier wait
 };
@@ -240,10 +243,7 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     bool dead = false;         // set after a wait timed out: later waits are skipped
 
     const int P = a.P;
-    const int pages_per_tile = P < kTile ? kTile / P : 1;
     const int tiles_per_page = P > kTile ? P / kTile : 1;
-    const int box_tok = P < kTile ? P : kTile;
-    const uint32_t box_bytes = (uint32_t)box_tok * 128u;
 
     auto page_id = [&](const Cursor &c, int pg) -> int {
         const int npages = (c.n + P - 1) / P;
@@ -270,44 +270,56 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const uint32_t bk = bars + st * 16, bv = bk + 8;
         int ids[4];
         int nbox = 1, tok_off = 0;
-        if (P < kTile) {
-            const int first = ic.tau * pages_per_tile;
-            const int npages = (ic.n + P - 1) / P;
-            nbox = npages - first < pages_per_tile ? npages - first : pages_per_tile;
+        if (a.box_tok > 0) {
+            // general path: boxes of box_tok <= min(P, 64) tokens; boxes that start at or past the end of
+            // the sequence are not fetched (their rows are masked, and zero-filled for V, below)
+            const int bt = a.box_tok;
+            const int t0 = ic.tau * kTile;
+            const int left = ic.n - t0;
+            nbox = left >= kTile ? (kTile >> a.lg_box) : ((left + bt - 1) >> a.lg_box);
 #pragma unroll
-            for (int b = 0; b < 4; ++b) ids[b] = (b < nbox) ? page_id(ic, first + b) : 0;
+            for (int b = 0; b < 4; ++b) ids[b] = (b < nbox) ? page_id(ic, (t0 + b * bt) >> a.lg_page) : 0;
         } else {
             ids[0] = page_id(ic, ic.tau / tiles_per_page);
             tok_off = (ic.tau % tiles_per_page) * kTile;
         }
-        if (lane == 0) {
-            if (P >= kTile) {
+        if (a.box_tok == 0) {
+            if (lane == 0) {
                 // one instruction per tile and pool: box = 64 tokens x all halves
                 const uint32_t bytes = (uint32_t)TB;
                 mbar_expect_tx(bk, bytes);
                 tma_load_5d(kdst, &tmK, 0, tok_off, 0, ic.g, ids[0], bk);
                 mbar_expect_tx(bv, bytes);
                 tma_load_5d(vdst, &tmV, 0, tok_off, 0, ic.g, ids[0], bv);
-            } else {
-                const uint32_t bytes = (uint32_t)nbox * box_bytes * HALVES;
-                const int c1 = a.tok_first ? 0 : ic.g;
-                const int c2 = a.tok_first ? ic.g : 0;
+            }
+        } else {
+            // lane = (pool, box, half): every box of the tile goes out in one warp instruction
+            const int bt = a.box_tok;
+            const uint32_t bbytes = (uint32_t)bt * 128u;
+            if (lane == 0) {
+                const uint32_t bytes = (uint32_t)nbox * bbytes * HALVES;
                 mbar_expect_tx(bk, bytes);
-#pragma unroll
-                for (int b = 0; b < 4; ++b)
-                    if (b < nbox) {
-#pragma unroll
-                        for (int h = 0; h < HALVES; ++h)
-                            tma_load_4d(kdst + h * (kTile * 128) + b * box_bytes, &tmK, h * 64, c1, c2, ids[b], bk);
-                    }
                 mbar_expect_tx(bv, bytes);
+            }
+            __syncwarp();
+            // lanes 0..7 = (pool, half, box parity): each issues boxes b and b + 2 of its pool and half,
+            // so a tile of 32-token boxes goes out in one warp instruction
+            const int is_v = lane >> 2, h = (lane >> 1) & 1, b0 = lane & 1;
+            if (lane < 8 && h < HALVES) {
+                const void *tm = is_v ? (const void *)&tmV : (const void *)&tmK;
+                const uint32_t dst = (is_v ? vdst : kdst) + h * (kTile * 128);
+                const uint32_t bar = is_v ? bv : bk;
 #pragma unroll
-                for (int b = 0; b < 4; ++b)
+                for (int x = 0; x < 2; ++x) {
+                    const int b = b0 + 2 * x;
                     if (b < nbox) {
-#pragma unroll
-                        for (int h = 0; h < HALVES; ++h)
-                            tma_load_4d(vdst + h * (kTile * 128) + b * box_bytes, &tmV, h * 64, c1, c2, ids[b], bv);
+                        const int id = b0 ? (x ? ids[3] : ids[1]) : (x ? ids[2] : ids[0]);
+                        const int off = (ic.tau * kTile + b * bt) & (P - 1);
+                        const int c1 = a.tok_first ? off : ic.g;
+                        const int c2 = a.tok_first ? ic.g : off;
+                        tma_load_4d(dst + b * bbytes, tm, h * 64, c1, c2, id, bar);
                     }
+                }
             }
         }
     };
@@ -814,13 +826,15 @@ static int check_params(const ts_attn_params *p)
 
 static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
-static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_params *p, int *tok_first)
+// box_tok = 0: one 5-D box per 64-token tile when the page holds a whole tile, else one 4-D box per page;
+// box_tok > 0: 4-D boxes of that many tokens (must divide 64 and not exceed the page size).
+static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_params *p, int *tok_first, int box_tok_req)
 {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return TS_ERR_CUDA;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r;
-    if (p->page_size >= kTile) {
+    if (p->page_size >= kTile && box_tok_req == 0) {
         // 5-D: (64 dims, token, 64-dim half, head, page).  One box = 64 tokens x all halves, laid out in
         // shared memory as [half][token][128 B]: a whole K or V tile per TMA instruction.
         *tok_first = 1;
@@ -834,13 +848,12 @@ static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_para
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         return r == CUDA_SUCCESS ? TS_OK : TS_ERR_UNSUPPORTED;
     }
-    // pages shorter than a tile: 4-D (64 dims, then {token, head} by ascending stride, page), one box
-    // per (page, half)
+    // 4-D (64 dims, then {token, head} by ascending stride, page), one box per (box_tok tokens, half)
     const bool tf = p->kv_token_stride <= p->kv_head_stride;
     *tok_first = tf ? 1 : 0;
     cuuint64_t dims[4], strides[3];
     cuuint32_t box[4];
-    const cuuint32_t box_tok = (cuuint32_t)p->page_size;
+    const cuuint32_t box_tok = box_tok_req > 0 ? (cuuint32_t)box_tok_req : (cuuint32_t)p->page_size;
     dims[0] = (cuuint64_t)p->head_dim;
     box[0] = 64;
     if (tf) {
@@ -951,6 +964,11 @@ static int launch_attn_tc(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs
     return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
+static bool use_tc_kernel(int D, int rows, float scale_log2)
+{
+    return D == 128 && rows > 16 && rows <= 128 && scale_log2 > 0.f && env_int("TS_ATTN_TC", 1) != 0;
+}
+
 template <int D>
 static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs &a, int sms, int smem_optin,
                          cudaStream_t stream, bool dry, int *ng)
@@ -958,7 +976,7 @@ static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv,
     // more than two n-tiles of rows at head_dim 128 and a positive scale: tcgen05 path (up to 16 rows
     // the warp-MMA kernel measures faster: 88 vs 73 % of the HBM peak on the bulk lengths at 16 rows);
     // TS_ATTN_TC=0 keeps the warp-MMA path for any row count
-    if (D == 128 && rows > 16 && rows <= 128 && a.scale_log2 > 0.f && env_int("TS_ATTN_TC", 1) != 0)
+    if (use_tc_kernel(D, rows, a.scale_log2))
         return launch_attn_tc(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 8) return launch_attn<D, 1, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 16) return launch_attn<D, 2, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
@@ -1000,11 +1018,24 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
 
+    // TMA box: the tcgen05 kernel takes a whole tile per instruction where the page allows it; the
+    // warp-MMA kernel takes boxes of TS_ATTN_BOX_TOK tokens (0 = a whole tile per instruction too)
+    const int rows_all = (p->num_q_heads / p->num_kv_heads) * p->q_len;
+    const float scale_log2 = p->scale * 1.4426950408889634f;
+    int box_tok = 0;
+    if (!use_tc_kernel(p->head_dim, rows_all, scale_log2)) {
+        // measured on the decode batches (one n-tile of rows): 32-token boxes, all issued by one warp
+        // instruction, stream 3-5 % faster than one box per tile; with more rows the issuing warp's
+        // extra instructions cost more than they gain
+        box_tok = env_int("TS_ATTN_BOX_TOK", (rows_all <= 8 && p->head_dim == 128) ? 32 : 0);
+        if (box_tok != 0 && box_tok != 16 && box_tok != 32 && box_tok != 64) box_tok = 0;
+        if (box_tok > p->page_size || (box_tok == 0 && p->page_size < kTile)) box_tok = p->page_size;
+    }
     CUtensorMap tk, tv;
     int tok_first = 1, tf2 = 1;
-    rc = make_tensor_map(&tk, k_pool, p, &tok_first);
+    rc = make_tensor_map(&tk, k_pool, p, &tok_first, box_tok);
     if (rc != TS_OK) return rc;
-    rc = make_tensor_map(&tv, v_pool, p, &tf2);
+    rc = make_tensor_map(&tv, v_pool, p, &tf2, box_tok);
     if (rc != TS_OK) return rc;
 
     AttnArgs a;
@@ -1023,7 +1054,12 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     a.G = p->num_q_heads / p->num_kv_heads; a.rows = a.G * p->q_len; a.P = p->page_size;
     a.max_pages = p->max_pages_per_seq; a.max_splits = max_splits; a.mode = mode;
     a.ngrp = 1; a.ns = 2; a.tok_first = tok_first;
-    a.scale_log2 = p->scale * 1.4426950408889634f;
+    a.box_tok = box_tok;
+    a.lg_page = 0;
+    while ((1 << a.lg_page) < p->page_size) ++a.lg_page;
+    a.lg_box = 0;
+    while ((1 << a.lg_box) < box_tok) ++a.lg_box;
+    a.scale_log2 = scale_log2;
     a.wait_cycles = (long long)dev.clock_khz * 2000LL;   // about two seconds of SM clocks
 
     // first pass fixes the launch geometry (NG) without launching
