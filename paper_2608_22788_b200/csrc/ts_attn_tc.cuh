@@ -438,26 +438,44 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         // tile it-2 before P of tile it is released (the PV of tile it cannot start earlier), and the PV
         // of the group's last tile at the end of the segment.
         auto wait_pv_done = [&](int t) { wait(obar(wg), (uint32_t)(t >> 1) & 1u); };
-        int it0 = 0, remaining = total;
+        // Q tile of pair (s_, g_) -> shared memory (K-major, 128-byte swizzle; rows past the tile are
+        // zero-filled): this thread's row, as asynchronous 16-byte copies.
+        auto issue_q = [&](int s_, int g_) {
+            const uint16_t *src = a.q + (((size_t)s_ * a.q_len + t_row) * a.Hq + (size_t)g_ * a.G + hl) * D;
+            const uint32_t qrow = base + kOffQ + (uint32_t)row * 128u;
+            const uint32_t nbytes = row_valid ? 16u : 0u;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const uint32_t addr = qrow + (uint32_t)(c >> 3) * 16384u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(addr), "l"(src + 8 * c), "r"(nbytes) : "memory");
+            }
+        };
+        // The copies of this thread have landed; make them visible to the tensor core and count the warp in.
+        auto publish_q = [&]() {
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(qfull);
+        };
+        int it0 = 0, remaining = total, seg_no = 0;
+        if (wg == 1 && remaining > 0) {
+            const Segment s0 = segment_at(cc, remaining, a);
+            issue_q(s0.s, s0.g);
+            publish_q();
+        }
         TS_TRACE_DECL
         while (remaining > 0) {
             const Segment sg = segment_at(cc, remaining, a);
-            if (wg == 0) {
-                // ---- Q tile -> shared memory (K-major, 128-byte swizzle), zero rows past the tile
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    a.q + (((size_t)sg.s * a.q_len + t_row) * a.Hq + (size_t)sg.g * a.G + hl) * D);
-                const uint32_t qrow = base + kOffQ + (uint32_t)row * 128u;
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (row_valid) v = __ldg(src + c);
-                    const uint32_t addr = qrow + (uint32_t)(c >> 3) * 16384u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(qfull);
+            const bool has_next = remaining > sg.len;
+            // Group 1 owns the Q tile: it fetches the next pair's while group 0 writes this pair's result.
+            Cursor nc = cc;
+            if (wg == 1 && has_next) {
+                nc.tau += sg.len - 1;
+                cur_advance(nc, a);
             }
+            // Group 1 may not hand the first P of a new segment to the PV issuer (which overwrites O1)
+            // before group 0 has read O1 of the previous segment: named barrier 3.
+            bool need_o_sync = (wg == 1 && seg_no > 0);
             float m_used = -INFINITY, l_sum = 0.f;
             const int lim = row_valid ? sg.n - a.q_len + t_row : -1;
             int last_t = -1;                              // last tile of this group in the segment
@@ -552,6 +570,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 fence_before_sync();
                 if (valid_tok < kTile) fence_proxy_async_smem();
                 __syncwarp();
+                if (need_o_sync) { named_bar_sync(3, 256); need_o_sync = false; }
                 if (lane == 0) mbar_arrive(pfull(buf));
                 if (q4 == 3 && lane == 0) TS_EVENT(it, 4)
                 l_sum = l_sum * alpha + rowsum;
@@ -559,11 +578,16 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
             // ---- end of the segment: merge the two groups' accumulators, write the result
             if (last_t >= 0) wait_pv_done(last_t);
+            if (need_o_sync) named_bar_sync(3, 256);      // no tile of this segment was ours: still pair up
             if (wg == 1) {
                 asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(stats), "f"(m_used), "f"(l_sum) : "memory");
                 fence_before_sync();
-                named_bar_sync(1, 256);
+                named_bar_sync(1, 256);       // every S = Q K^T and P V of the segment has completed
                 named_bar_sync(2, 256);       // group 0 has read the statistics: the slot may be rewritten
+                if (has_next) {
+                    issue_q(nc.s, nc.g);       // the tile is free: every Q K^T of the segment is done
+                    publish_q();
+                }
             } else {
                 named_bar_sync(1, 256);
                 fence_after_sync();
@@ -626,9 +650,11 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         }
                     }
                 }
-                if (row_valid && !write_final) *pl = L > 0.f ? (Mref + log2f(L)) * 0.6931471805599453f : -INFINITY;
                 fence_before_sync();
+                if (has_next) asm volatile("bar.arrive 3, 256;" ::: "memory");   // O0 and O1 have been read
+                if (row_valid && !write_final) *pl = L > 0.f ? (Mref + log2f(L)) * 0.6931471805599453f : -INFINITY;
             }
+            ++seg_no;
             it0 += sg.len;
             remaining -= sg.len;
             cc.tau += sg.len - 1;
