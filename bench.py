@@ -41,7 +41,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, decode attention kernel, from the
 # ncu capture summarised in profiles/ts_attn_kernel_decode_bulk64.md (traffic grows with the KV bytes)
-NCU_TRAFFIC_RATIO_DECODE = 1.025
+NCU_TRAFFIC_RATIO_DECODE = 1.013
 
 
 def measured_peaks():
@@ -565,6 +565,22 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
                {"emitted_tokens": semitted, "temperature": 0.7, "top_k": 20, "top_p": 0.8,
                 "note": "drafts = row argmax up to the seeded cut point; acceptance is stochastic here"})
         del acc, smp
+
+    # route-specific draft depths (Section 4.3: a shallow depth on the wide bulk pool, a deep one on the
+    # narrow tail pool, the two summing to twice the base depth): verify attention on the bulk batch
+    # (256 sequences) and on the tail-replica batch (16 sequences) at depths 3, 4 and 5
+    depth = {}
+    for route, lens in (("bulk", wl.lens_bulk(seed)), ("tail", wl.lens_verify(seed))):
+        for g in (3, 4, 5):
+            dw = Workload(f"{route}_verify_g{g}", lens, pool, q_len=1 + g, seed=seed + 20 + g)
+            med, mn = time_with_flush(dw.attn, flush, iters=5, warmup=2)
+            assert dw.status() == 0
+            depth[f"{route}_g{g}"] = {"ms": med, "positions_per_s": dw.b.num_seqs * (1 + g) / (med * 1e-3),
+                                      "GBps": gbs(dw.bytes, med), "frac_of_measured_peak": gbs(dw.bytes, med) / peak}
+            del dw
+    depth["pairs_ms"] = {f"bulk{gb}+tail{gt}": depth[f"bulk_g{gb}"]["ms"] + depth[f"tail_g{gt}"]["ms"]
+                         for gb, gt in ((3, 5), (4, 4), (5, 3))}
+    out["depth_pairs:ts_verify_attn"] = depth
 
     # concurrency sweep on the mixed length pool: attention-only analogue of v(b) and b*v(b)
     pool_lens = wl.lens_mixed(seed)
