@@ -149,7 +149,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int b_mn_major)
 // -DTS_TC_TRACE; sums of SM clock cycles land in the 16 x 8-byte words after the status word.
 #ifdef TS_TC_TRACE
 // absolute timestamps of pipeline events of tiles 200..207 of CTA 0 (event e of tile t at ev[(t-200)*8 + e])
-#define TS_EVENT(t, e) { if (blockIdx.x == 0 && (t) >= 200 && (t) < 208) reinterpret_cast<long long *>(a.part_o)[((t) - 200) * 8 + (e)] = clock64(); }
+#define TS_EVENT(t, e) { if (blockIdx.x == 0 && (t) >= 200 && (t) < 208) reinterpret_cast<long long *>(a.part_o)[((t) - 200) * 16 + (e)] = clock64(); }
 #define TS_TRACE_DECL long long tr_t = clock64(), tr_acc[6] = {0, 0, 0, 0, 0, 0};
 #define TS_TRACE(i) { const long long tr_n = clock64(); tr_acc[i] += tr_n - tr_t; tr_t = tr_n; }
 #else
@@ -487,6 +487,13 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const int buf = (wg << 1) | ((it >> 1) & 1);
                 const uint32_t sp_tmem = tmem_base + tlane + (uint32_t)buf * 64;
                 TS_TRACE(0)
+                if (wg == 1 && has_next && j + 2 >= sg.len && row_valid) {
+                    // last tile of this group in the segment: pull the next pair's Q rows into L2, so that the
+                    // copy at the end of the segment does not wait for HBM
+                    const uint16_t *src = a.q + (((size_t)nc.s * a.q_len + t_row) * a.Hq + (size_t)nc.g * a.G + hl) * D;
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src + 64));
+                }
                 wait(sfull(buf), (uint32_t)(it >> 2) & 1u);
                 fence_after_sync();
                 TS_TRACE(1)
@@ -578,6 +585,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             }
             // ---- end of the segment: merge the two groups' accumulators, write the result
             if (last_t >= 0) wait_pv_done(last_t);
+            if (q4 == 3 && lane == 0) TS_EVENT(it0 + sg.len - 1, 8 + wg)
             if (need_o_sync) named_bar_sync(3, 256);      // no tile of this segment was ours: still pair up
             if (wg == 1) {
                 asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(stats), "f"(m_used), "f"(l_sum) : "memory");
@@ -587,6 +595,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 if (has_next) {
                     issue_q(nc.s, nc.g);       // the tile is free: every Q K^T of the segment is done
                     publish_q();
+                    if (q4 == 0 && lane == 0) TS_EVENT(it0 + sg.len - 1, 10)
                 }
             } else {
                 named_bar_sync(1, 256);
@@ -652,6 +661,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 }
                 fence_before_sync();
                 if (has_next) asm volatile("bar.arrive 3, 256;" ::: "memory");   // O0 and O1 have been read
+                if (q4 == 3 && lane == 0) TS_EVENT(it0 + sg.len - 1, 11)
                 if (row_valid && !write_final) *pl = L > 0.f ? (Mref + log2f(L)) * 0.6931471805599453f : -INFINITY;
             }
             ++seg_no;
