@@ -197,7 +197,6 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t bsf = bar0 + 8u * (3 * kStages);
     auto sfull = [&](int b) { return bsf + 8u * b; };            // per S/P buffer (4)
     auto pfull = [&](int b) { return bsf + 8u * (4 + b); };      // per S/P buffer (4)
-    auto obar = [&](int w) { return bsf + 8u * (8 + w); };       // per softmax group (2)
     const uint32_t qfull = bsf + 8u * 10;
     auto pdone = [&](int b) { return bsf + 8u * (11 + b); };     // per S/P buffer (4): its PV has finished
     const uint32_t tmem_slot = bsf + 8u * 15;
@@ -210,7 +209,6 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     if (warp == 0 && lane == 0) {
         for (int st = 0; st < kStages; ++st) { mbar_init(kfull(st), 1); mbar_init(vfull(st), 1); mbar_init(kvfree(st), 1); }
         for (int b = 0; b < 4; ++b) { mbar_init(sfull(b), 1); mbar_init(pfull(b), 4); mbar_init(pdone(b), 1); }
-        for (int w = 0; w < 2; ++w) mbar_init(obar(w), 1);
         mbar_init(qfull, 4);
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
@@ -403,7 +401,6 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                             umma_bf16_ts(o_tmem, p_tmem + part * 32 + ks * 8, bd, idesc_pv, (first && part == 0 && ks == 0) ? 0u : 1u);
                         }
                     umma_commit(pdone(buf));
-                    umma_commit(obar(w));
                     umma_commit(kvfree(st));
                     TS_TRACE(5)
                     TS_EVENT(t, 6)
@@ -433,11 +430,19 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const int tid_wg = (threadIdx.x - 96) & 127;      // 0..127 inside the group
         const uint32_t o_col = kTmemO + (uint32_t)wg * 128u;
         const uint32_t stats = base + kOffStats + (uint32_t)row * 8u;
-        // Wait until this group's PV of tile t (parity wg) has finished.  A parity wait only tells the
-        // current phase from the previous one, so every phase of obar[wg] is observed in order: the PV of
-        // tile it-2 before P of tile it is released (the PV of tile it cannot start earlier), and the PV
-        // of the group's last tile at the end of the segment.
-        auto wait_pv_done = [&](int t) { wait(obar(wg), (uint32_t)(t >> 1) & 1u); };
+        // This group's PVs are numbered u = it >> 1; PV u signals pdone of buffer 2*wg + (u & 1), phase u >> 1.
+        // A parity wait only tells the current phase from the previous one, so the phases of each of the two
+        // barriers are observed in order, and PV u - 2 (the previous phase of the barrier PV u will signal) is
+        // observed before P of tile u is released: PV u cannot complete earlier.  That is all the common tile
+        // waits for: its P is released while PV u - 1 may still be running (the tensor core accumulates in
+        // issue order).  Only a rescale of O, and the end of a segment, wait for every PV issued so far.
+        int seen = 0;                                     // PVs of this group observed so far
+        auto observe_upto = [&](int u_target) {
+            while (seen <= u_target) {
+                wait(pdone((wg << 1) | (seen & 1)), (uint32_t)(seen >> 1) & 1u);
+                ++seen;
+            }
+        };
         // Q tile of pair (s_, g_) -> shared memory (K-major, 128-byte swizzle; rows past the tile are
         // zero-filled): this thread's row, as asynchronous 16-byte copies.
         auto issue_q = [&](int s_, int g_) {
@@ -557,10 +562,11 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 }
-                // the PV of this group's previous tile (it-2), the last one that accumulated into its O
-                if (it >= 2) wait_pv_done(it - 2);
-                // lazy rescale of this group's O in TMEM (warp-collective)
+                const int u = it >> 1;
+                if (u >= 2) observe_upto(u - 2);
+                // lazy rescale of this group's O in TMEM (warp-collective): every PV into it must have finished
                 if (__any_sync(FULL, rescale)) {
+                    observe_upto(u - 1);
                     fence_after_sync();
                     const float f = rescale ? alpha : 1.f;
 #pragma unroll 1
@@ -584,7 +590,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 TS_TRACE(5)
             }
             // ---- end of the segment: merge the two groups' accumulators, write the result
-            if (last_t >= 0) wait_pv_done(last_t);
+            if (last_t >= 0) observe_upto(last_t >> 1);
             if (q4 == 3 && lane == 0) TS_EVENT(it0 + sg.len - 1, 8 + wg)
             if (need_o_sync) named_bar_sync(3, 256);      // no tile of this segment was ours: still pair up
             if (wg == 1) {
