@@ -60,6 +60,9 @@ def _load():
         lib.ora_accept_sample.argtypes = [c_u16p, ctypes.c_int64, c_i32p, c_f64p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
                                           c_i32p, c_i32p, c_i32p, c_f64p]
+        lib.ora_rope.restype = ctypes.c_int
+        lib.ora_rope.argtypes = [c_u16p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_float),
+                                 ctypes.c_int64, ctypes.c_int, ctypes.c_int, c_f64p]
         lib.ora_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -180,3 +183,22 @@ def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, to
     if rc != 0:
         raise RuntimeError(f"ora_accept_sample failed ({rc})")
     return acc, out, ids, pp
+
+
+def rope(x, pos, inv_freq):
+    """Rotary position embedding ("rotate-half" pairing) of bf16 rows.
+
+    ``x``: uint16 bf16 bits ``[rows, heads, D]``; ``pos``: int ``[rows]``; ``inv_freq``: float32
+    ``[D/2]``.  Returns float64 ``[rows, heads, D]`` (not rounded).
+    """
+    lib = _load()
+    x = np.ascontiguousarray(x, dtype=np.uint16)
+    rows, heads, D = x.shape
+    pos = np.ascontiguousarray(pos, dtype=np.int64).reshape(rows)
+    f = np.ascontiguousarray(inv_freq, dtype=np.float32).reshape(D // 2)
+    out = np.empty((rows, heads, D), dtype=np.float64)
+    rc = lib.ora_rope(_p(x, ctypes.c_uint16), _p(pos, ctypes.c_int64), _p(f, ctypes.c_float), rows, heads, D,
+                      _p(out, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError(f"ora_rope failed ({rc})")
+    return out

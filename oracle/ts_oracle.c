@@ -28,6 +28,11 @@
  *                        regime (temperature, top-k, top-p; Appendix, Table
  *                        "shared-sampling-config") with point-proposal drafts.
  *
+ *   ora_rope             rotary position embedding of the step's query and key
+ *                        rows ("rotate-half" pairing, the form the Qwen models
+ *                        the paper evaluates use; the paper itself prints no
+ *                        formula for it): the step before attention.
+ *
  * All bf16 inputs are uint16 bit patterns, decoded exactly to double.
  * Pins for every function live in tests/test_oracle_*.py (brute force on
  * unpaged tensors written independently in NumPy, closed forms, invariants).
@@ -320,5 +325,34 @@ int ora_accept_sample(const uint16_t *logits, int64_t row_stride, const int32_t 
         }
         accept_len[b] = a;
     }
+    return 0;
+}
+
+/*
+ * Rotary position embedding, "rotate-half" pairing: dimension d < D/2 is paired with d + D/2,
+ *   angle  = pos * inv_freq[d]                  (pos integer, inv_freq given as float, product in double)
+ *   out[d]       = x[d] * cos(angle) - x[d + D/2] * sin(angle)
+ *   out[d + D/2] = x[d + D/2] * cos(angle) + x[d] * sin(angle)
+ * i.e. the complex number x[d] + i x[d + D/2] times exp(i angle).
+ *   x    bf16 bits [rows, heads, D]      pos  int64 [rows]      inv_freq  float [D/2]
+ *   out  double [rows, heads, D], not rounded
+ */
+int ora_rope(const uint16_t *x, const int64_t *pos, const float *inv_freq, int64_t rows, int heads, int D,
+             double *out)
+{
+    if (!x || !pos || !inv_freq || !out || rows < 0 || heads < 1 || D < 2 || (D & 1)) return -1;
+    const int half = D / 2;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int h = 0; h < heads; ++h) {
+            const uint16_t *xr = x + (r * heads + h) * (int64_t)D;
+            double *o = out + (r * heads + h) * (int64_t)D;
+            for (int d = 0; d < half; ++d) {
+                const double angle = (double)pos[r] * (double)inv_freq[d];
+                const double c = cos(angle), sn = sin(angle);
+                const double a = bf16_to_double(xr[d]), b = bf16_to_double(xr[d + half]);
+                o[d] = a * c - b * sn;
+                o[d + half] = b * c + a * sn;
+            }
+        }
     return 0;
 }
