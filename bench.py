@@ -545,6 +545,21 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
     record("tail:ts_decode_attn_splitkv+ts_lse_merge", w.bytes, med, mn, w.b.num_seqs,
            {"max_splits": S, "num_splits": ns.cpu().tolist()})
 
+    # the step before attention: rotary embedding of the step's Q and K rows fused with the K/V append
+    # (the bulk batch appends 256 rows, the verify batch at gamma 16 appends 272)
+    inv_freq = torch.from_numpy((1.0e6 ** (-np.arange(0, 128, 2, dtype=np.float64) / 128)).astype(np.float32)).cuda()
+    for name in ("bulk", "verify_g16"):
+        w = W[name]
+        nk = torch.from_numpy(wl.normal_bf16((w.b.num_seqs, w.b.q_len, 8, 128), seed=seed + 31).view(np.int16)).cuda().view(torch.bfloat16)
+        nv = torch.from_numpy(wl.normal_bf16((w.b.num_seqs, w.b.q_len, 8, 128), seed=seed + 32).view(np.int16)).cuda().view(torch.bfloat16)
+        q_rot = torch.empty_like(w.q)
+        med, mn = time_with_flush(lambda: api.ts_rope_kv_append(w.geom, w.q, q_rot, nk, nv, pool.k, pool.v, w.bt, w.lens,
+                                                                inv_freq), flush)
+        rows = w.b.num_seqs * w.b.q_len
+        nbytes = rows * (2 * 32 + 4 * 8) * 128 * 2       # q in + out, k and v in + out
+        record(f"{name}:ts_rope_kv_append", nbytes, med, mn, rows, {"rows": rows})
+        del nk, nv, q_rot
+
     # speculative verify: attention, then greedy acceptance
     for g in (4, 8, 16):
         w = W[f"verify_g{g}"]

@@ -152,6 +152,27 @@ int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *parti
 int ts_kv_append(const ts_attn_params *p, const void *new_k, const void *new_v, void *k_pool, void *v_pool,
                  const int32_t *block_table, const int32_t *kv_lens, void *stream);
 
+/*
+ * ts_kv_append with the rotary position embedding of the step's query and key rows fused in: the
+ * step before attention in the models the paper serves (Qwen3 family, Section 4.1); the paper itself
+ * prints no formula for it, so the convention is fixed here.  "Rotate-half" pairing: with
+ * angle = pos * inv_freq[d] for d < head_dim / 2 and pos = kv_lens[s] - q_len + t,
+ *   y[d]              = x[d] * cos(angle) - x[d + head_dim/2] * sin(angle)
+ *   y[d + head_dim/2] = x[d + head_dim/2] * cos(angle) + x[d] * sin(angle)
+ * computed in fp32 from the bf16 inputs (the angle itself in double, reduced mod 2 pi before the
+ * float sincos), rounded to bf16 (nearest even).
+ *   q_in      bf16 [num_seqs, q_len, num_q_heads, head_dim]  -> rotated into q_out (same shape; q_out
+ *             may be q_in: each element pair is read and written by one thread)
+ *   new_k     bf16 [num_seqs, q_len, num_kv_heads, head_dim] -> rotated, written into k_pool
+ *   new_v     same shape, copied bit for bit into v_pool
+ *   inv_freq  float [head_dim / 2], device (a model constant, e.g. base^(-2d/head_dim))
+ * Placement, skipping of negative positions, strides and alignment as in ts_kv_append;
+ * head_dim % 16 == 0 and head_dim <= 256.  Errors are detected on the host before the launch.
+ */
+int ts_rope_kv_append(const ts_attn_params *p, const void *q_in, void *q_out, const void *new_k,
+                      const void *new_v, void *k_pool, void *v_pool, const int32_t *block_table,
+                      const int32_t *kv_lens, const float *inv_freq, void *stream);
+
 /* Scratch bytes for ts_accept_greedy (host-only; 0 for invalid sizes). */
 size_t ts_accept_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab);
 

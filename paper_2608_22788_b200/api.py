@@ -22,7 +22,7 @@ TS_OK = 0
 EXPORTED_SYMBOLS = (
     "ts_attn_workspace_bytes", "ts_splitkv_workspace_bytes", "ts_decode_attn", "ts_verify_attn",
     "ts_decode_attn_splitkv", "ts_lse_merge", "ts_accept_workspace_bytes", "ts_accept_greedy",
-    "ts_accept_greedy_noalloc", "ts_sample_workspace_bytes", "ts_accept_sample", "ts_kv_append",
+    "ts_accept_greedy_noalloc", "ts_sample_workspace_bytes", "ts_accept_sample", "ts_kv_append", "ts_rope_kv_append",
     "ts_set_attn_timing_events", "ts_status_string",
 )
 
@@ -79,6 +79,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ts_accept_sample.argtypes = [vp, i64, vp, vp, i32, i32, i32, ctypes.c_float, i32, ctypes.c_float, vp, vp, vp, sz, vp]
     lib.ts_kv_append.restype = ctypes.c_int
     lib.ts_kv_append.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
+    lib.ts_rope_kv_append.restype = ctypes.c_int
+    lib.ts_rope_kv_append.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ts_set_attn_timing_events.restype = ctypes.c_int
     lib.ts_set_attn_timing_events.argtypes = [vp, vp]
     lib.ts_status_string.restype = ctypes.c_char_p
@@ -263,3 +265,15 @@ def ts_kv_append(geom, new_k, new_v, k_pool, v_pool, block_table, kv_lens):
     rc = lib.ts_kv_append(ctypes.byref(p), _ptr(new_k, "new_k"), _ptr(new_v, "new_v"), _ptr(k_pool, "k_pool"),
                           _ptr(v_pool, "v_pool"), _ptr(block_table, "block_table"), _ptr(kv_lens, "kv_lens"), _stream())
     _check(rc, "ts_kv_append")
+
+
+def ts_rope_kv_append(geom, q_in, q_out, new_k, new_v, k_pool, v_pool, block_table, kv_lens, inv_freq):
+    """Rotate this step's Q rows (into ``q_out``) and K rows with the rotary embedding of their
+    positions, and write the rotated K and the V rows into the paged pools (before attention)."""
+    lib = load_library()
+    p = geom.c_struct()
+    rc = lib.ts_rope_kv_append(ctypes.byref(p), _ptr(q_in, "q_in"), _ptr(q_out, "q_out"), _ptr(new_k, "new_k"),
+                               _ptr(new_v, "new_v"), _ptr(k_pool, "k_pool"), _ptr(v_pool, "v_pool"),
+                               _ptr(block_table, "block_table"), _ptr(kv_lens, "kv_lens"), _ptr(inv_freq, "inv_freq"),
+                               _stream())
+    _check(rc, "ts_rope_kv_append")
