@@ -59,7 +59,8 @@ def _load():
         lib.ora_accept_sample.restype = ctypes.c_int
         lib.ora_accept_sample.argtypes = [c_u16p, ctypes.c_int64, c_i32p, c_f64p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
-                                          c_i32p, c_i32p, c_i32p, c_f64p]
+                                          c_i32p, c_i32p, c_i32p, c_f64p, ctypes.POINTER(ctypes.c_uint8),
+                                          ctypes.c_int64, ctypes.c_double]
         lib.ora_rope.restype = ctypes.c_int
         lib.ora_rope.argtypes = [c_u16p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_float),
                                  ctypes.c_int64, ctypes.c_int, ctypes.c_int, c_f64p]
@@ -159,12 +160,17 @@ def accept_greedy(logits, draft, nthreads: int = 0):
     return tgt, acc, out
 
 
-def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, top_p: float):
+def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, top_p: float,
+                  seen=None, presence_penalty: float = 0.0):
     """Lossless acceptance under temperature / top-k / top-p sampling with point-proposal drafts.
 
     ``logits``: uint16 bf16 bits ``[B, gamma+1, V]``; ``draft``: int ``[B, gamma]``; ``uniforms``:
     float ``[B, gamma+1, 2]`` in [0, 1).  Returns ``(accept_len [B], out_tokens [B,gamma+1],
     kept_ids [B,gamma+1,top_k], kept_p [B,gamma+1,top_k])``.
+
+    ``seen``: optional uint8 bitmap ``[B, >= ceil(V/8)]`` (bit ``v & 7`` of byte ``v >> 3``) of the
+    tokens each sequence has generated so far; with ``presence_penalty`` their logits, and those of
+    the earlier drafts of the block, are lowered by the penalty before the top-k selection.
     """
     lib = _load()
     logits = np.ascontiguousarray(logits, dtype=np.uint16)
@@ -172,6 +178,11 @@ def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, to
     gamma = R - 1
     draft = np.ascontiguousarray(draft, dtype=np.int32).reshape(B, gamma)
     u = np.ascontiguousarray(uniforms, dtype=np.float64).reshape(B, R, 2)
+    sb, sstride = None, 0
+    if seen is not None:
+        sb = np.ascontiguousarray(seen, dtype=np.uint8)
+        assert sb.ndim == 2 and sb.shape[0] == B and sb.shape[1] * 8 >= V
+        sstride = sb.shape[1]
     acc = np.empty((B,), dtype=np.int32)
     out = np.empty((B, R), dtype=np.int32)
     ids = np.empty((B, R, top_k), dtype=np.int32)
@@ -179,7 +190,7 @@ def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, to
     rc = lib.ora_accept_sample(_p(logits, ctypes.c_uint16), V, _p(draft, ctypes.c_int32), _p(u, ctypes.c_double),
                                B, gamma, V, float(temperature), int(top_k), float(top_p),
                                _p(acc, ctypes.c_int32), _p(out, ctypes.c_int32), _p(ids, ctypes.c_int32),
-                               _p(pp, ctypes.c_double))
+                               _p(pp, ctypes.c_double), _p(sb, ctypes.c_uint8), int(sstride), float(presence_penalty))
     if rc != 0:
         raise RuntimeError(f"ora_accept_sample failed ({rc})")
     return acc, out, ids, pp

@@ -257,24 +257,43 @@ int ora_max_threads(void)
  *
  * The probabilities of every row are also returned (kept_ids / kept_p, top_k slots per row, -1 / 0
  * padded) so that tests can tell a wrong decision from one where u falls within rounding of p.
+ *
+ * Presence penalty (the same table lists 1.5): before step 1 the logit of every token that is
+ * "present" for row (b, i) is lowered by the penalty, once, however often the token occurred:
+ *   present(b, i) = tokens whose bit is set in seen[b] (bit v & 7 of byte v >> 3: what sequence b
+ *                   has generated before this step; the caller keeps it)  union  draft[b, 0 .. i-1]
+ *                   (row i is conditioned on those drafts having been accepted).
+ * The subtraction is done in single precision on the decoded logit (the precision in which a
+ * serving engine holds its logits when it applies penalties).  seen == NULL: nothing seen yet.
  */
 int ora_accept_sample(const uint16_t *logits, int64_t row_stride, const int32_t *draft,
                       const double *uniforms /* [B, gamma+1, 2] */, int B, int gamma, int V,
                       double temperature, int top_k, double top_p, int32_t *accept_len,
                       int32_t *out_tokens, int32_t *kept_ids /* [B, gamma+1, top_k] */,
-                      double *kept_p /* [B, gamma+1, top_k] */)
+                      double *kept_p /* [B, gamma+1, top_k] */, const uint8_t *seen,
+                      int64_t seen_stride, double presence_penalty)
 {
     if (B < 0 || gamma < 0 || V <= 0 || top_k < 1 || !(temperature > 0.0)) return -1;
     const int R = gamma + 1;
+    const float pen = (float)presence_penalty;
     for (int r = 0; r < B * R; ++r) {
         const uint16_t *row = logits + (int64_t)r * row_stride;
+        const int b = r / R, i = r % R;
         int32_t *ids = kept_ids + (int64_t)r * top_k;
         double *pp = kept_p + (int64_t)r * top_k;
         double val[top_k];
         int n = 0;
         /* step 1: insertion into a list sorted by (value descending, index ascending) */
         for (int v = 0; v < V; ++v) {
-            const double x = bf16_to_double(row[v]);
+            double x = bf16_to_double(row[v]);
+            if (pen != 0.0f) {
+                int present = seen ? (seen[(int64_t)b * seen_stride + (v >> 3)] >> (v & 7)) & 1 : 0;
+                for (int j = 0; j < i && !present; ++j) present = draft[(int64_t)b * gamma + j] == v;
+                if (present) {
+                    volatile float y = (float)x - pen;      /* one single-precision subtraction */
+                    x = (double)y;
+                }
+            }
             if (x != x) continue;                       /* NaN */
             if (n == top_k && !(x > val[n - 1])) continue;   /* not better than the worst kept (ties lose: higher index) */
             int pos = n < top_k ? n : top_k - 1;

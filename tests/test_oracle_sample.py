@@ -149,3 +149,78 @@ def test_nan_never_a_candidate_and_masked_vocabulary():
     assert ids[0, 0, :2].tolist() == [7, 8] and 3 not in ids[0, 0]
     assert np.allclose(pp[0, 0, :2], [0.5, 0.5]) and np.allclose(pp[0, 0, 2:], 0)
     assert out[0, 0] == 8 and acc[0] == 0
+
+
+# ------------------------------------------------------------------------------------------------
+# presence penalty
+# ------------------------------------------------------------------------------------------------
+def _bitmap(B, V, tokens_per_seq):
+    bm = np.zeros((B, (V + 7) // 8), np.uint8)
+    for b, toks in enumerate(tokens_per_seq):
+        for v in toks:
+            bm[b, v >> 3] |= np.uint8(1 << (v & 7))
+    return bm
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_presence_penalty_equals_plain_run_on_prepenalised_logits(seed):
+    # logits on a grid of halves and a penalty of 1.5: every penalised value is again a bf16 number, so the
+    # penalised call must equal the plain call on logits lowered beforehand, row by row, with row i also
+    # lowering the drafts 0 .. i-1 (built here with NumPy, independently of the oracle's own loop)
+    rng = np.random.default_rng(100 + seed)
+    B, gamma, V = 4, 3, 160
+    grid = (rng.integers(-24, 25, (B, gamma + 1, V)) * 0.5).astype(np.float32)
+    logits = _bits(grid)
+    draft = rng.integers(0, V, (B, gamma)).astype(np.int32)
+    draft[0, 1] = draft[0, 0]                                   # a repeated draft is penalised once
+    seen_tokens = [sorted(set(rng.integers(0, V, 30).tolist())) for _ in range(B)]
+    seen_tokens[1].append(int(draft[1, 0]))                     # seen and drafted: still penalised once
+    bm = _bitmap(B, V, seen_tokens)
+    u = rng.random((B, gamma + 1, 2))
+    T, k, pnuc, pen = 0.7, 20, 0.8, 1.5
+    got = oracle.accept_sample(logits, draft, u, temperature=T, top_k=k, top_p=pnuc, seen=bm, presence_penalty=pen)
+    lowered = grid.copy()
+    for b in range(B):
+        for i in range(gamma + 1):
+            present = set(seen_tokens[b]) | set(int(x) for x in draft[b, :i])
+            for v in present:
+                lowered[b, i, v] -= pen
+    assert np.array_equal(wl.bf16_bits_to_f32(_bits(lowered)), lowered)       # exactly representable
+    want = oracle.accept_sample(_bits(lowered), draft, u, temperature=T, top_k=k, top_p=pnuc)
+    for g, w in zip(got, want):
+        assert np.array_equal(g, w)
+    racc, rout = brute_accept(_bits(lowered), draft, u, T, k, pnuc)
+    assert np.array_equal(got[0], racc) and np.array_equal(got[1], rout)
+
+
+def test_presence_penalty_zero_or_nothing_present_changes_nothing():
+    rng = np.random.default_rng(7)
+    B, gamma, V = 3, 0, 500
+    logits = wl.make_logits(B, gamma, V, seed=9)
+    draft = np.zeros((B, 0), np.int32)
+    u = rng.random((B, 1, 2))
+    base = oracle.accept_sample(logits, draft, u, temperature=0.7, top_k=20, top_p=0.8)
+    bm = _bitmap(B, V, [[1, 2, 3]] * B)
+    same = oracle.accept_sample(logits, draft, u, temperature=0.7, top_k=20, top_p=0.8, seen=bm, presence_penalty=0.0)
+    empty = oracle.accept_sample(logits, draft, u, temperature=0.7, top_k=20, top_p=0.8,
+                                 seen=np.zeros_like(bm), presence_penalty=1.5)
+    for a, b_, c in zip(base, same, empty):
+        assert np.array_equal(a, b_) and np.array_equal(a, c)
+
+
+def test_large_presence_penalty_removes_seen_tokens_from_the_kept_set():
+    rng = np.random.default_rng(8)
+    B, gamma, V = 2, 2, 300
+    logits = wl.make_logits(B, gamma, V, seed=10)
+    f = wl.bf16_bits_to_f32(logits)
+    top = np.argsort(-f, axis=-1)[..., :5]                      # the five best tokens of every row
+    seen_tokens = [sorted(set(top[b].reshape(-1).tolist())) for b in range(B)]
+    bm = _bitmap(B, V, seen_tokens)
+    draft = top[:, :gamma, 0].astype(np.int32)
+    u = rng.random((B, gamma + 1, 2))
+    acc, out, ids, pp = oracle.accept_sample(logits, draft, u, temperature=0.7, top_k=20, top_p=0.8,
+                                             seen=bm, presence_penalty=1000.0)
+    for b in range(B):
+        kept = set(ids[b][ids[b] >= 0].tolist())
+        assert not (kept & set(seen_tokens[b]))
+        assert acc[b] == 0                                      # the drafts are seen tokens: never kept, rejected
