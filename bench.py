@@ -202,11 +202,17 @@ class Accept:
 class Sample:
     """ts_accept_sample on the same logits / drafts as an Accept instance (paper's sampling regime)."""
 
-    def __init__(self, acc: "Accept", seed=0, temperature=0.7, top_k=20, top_p=0.8):
+    def __init__(self, acc: "Accept", seed=0, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=0.0,
+                 seen_density=0.0):
         import torch
         self.api, self.acc = acc.api, acc
         self.kw = dict(temperature=temperature, top_k=top_k, top_p=top_p)
         rng = np.random.default_rng([seed, 17])
+        if presence_penalty != 0.0:
+            # seen-token bitmap: each sequence has generated `seen_density` of the vocabulary so far
+            bits = np.random.default_rng([seed, 18]).random((acc.B, acc.V)) < seen_density
+            self.kw.update(presence_penalty=presence_penalty,
+                           seen=torch.from_numpy(np.packbits(bits, axis=1, bitorder="little")).cuda())
         self.u = torch.from_numpy(rng.random((acc.B, acc.gamma + 1, 2), dtype=np.float32)).cuda()
         self.alen = torch.empty((acc.B,), dtype=torch.int32, device="cuda")
         self.tok = torch.empty((acc.B, acc.gamma + 1), dtype=torch.int32, device="cuda")
@@ -579,7 +585,12 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         record(f"verify_g{g}:ts_accept_sample", acc.bytes, smed, smn, semitted,
                {"emitted_tokens": semitted, "temperature": 0.7, "top_k": 20, "top_p": 0.8,
                 "note": "drafts = row argmax up to the seeded cut point; acceptance is stochastic here"})
-        del acc, smp
+        pen = Sample(acc, seed=seed, presence_penalty=1.5, seen_density=0.03)
+        pmed, pmn = time_with_flush(pen.run, flush)
+        record(f"verify_g{g}:ts_accept_sample_penalized", acc.bytes, pmed, pmn, int((pen.alen + 1).sum().item()),
+               {"temperature": 0.7, "top_k": 20, "top_p": 0.8, "presence_penalty": 1.5,
+                "note": "seen-token bitmap with 3 % of the vocabulary set (about 4500 distinct generated tokens)"})
+        del acc, smp, pen
 
     # route-specific draft depths (Section 4.3: a shallow depth on the wide bulk pool, a deep one on the
     # narrow tail pool, the two summing to twice the base depth): verify attention on the bulk batch

@@ -217,13 +217,29 @@ size_t ts_sample_workspace_bytes(int32_t num_seqs, int32_t gamma, int32_t vocab,
  *   workspace   >= ts_sample_workspace_bytes(...) bytes, clobbered
  * temperature > 0, 1 <= top_k <= 32, 0 < top_p <= 1, vocab <= 524288.  Token selection is exact;
  * probabilities are fp32, so a uniform within rounding of a probability may decide either way.
- * Penalties on already generated tokens (the paper's presence penalty) are the caller's job: apply
- * them to the logits first.
+ * Penalties on already generated tokens: see ts_accept_sample_penalized below.
  */
 int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draft, const float *uniforms,
                      int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k,
                      float top_p, int32_t *accept_len, int32_t *out_tokens, void *workspace,
                      size_t workspace_bytes, void *stream);
+
+/*
+ * ts_accept_sample with the presence penalty of the same sampling table (1.5 there): before the top-k
+ * selection of row (b, i) the logit of every token that is present for that row is lowered by
+ * presence_penalty, once however often the token occurred.  Present for row (b, i):
+ *   the tokens whose bit is set in seen[b] (bit v & 7 of byte seen[b * seen_stride + (v >> 3)]): what
+ *   sequence b has generated before this step, kept by the caller (device memory, may be NULL);
+ *   and draft[b, 0 .. i-1], on whose acceptance row i is conditioned.
+ * The subtraction is one fp32 operation on the decoded logit; selection stays exact on those values.
+ * seen_stride (bytes per sequence) * 8 >= vocab.  presence_penalty = 0, or no bitmap and gamma = 0,
+ * is ts_accept_sample exactly.  Everything else as ts_accept_sample.
+ */
+int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int32_t *draft,
+                               const float *uniforms, int32_t num_seqs, int32_t gamma, int32_t vocab,
+                               float temperature, int32_t top_k, float top_p, float presence_penalty,
+                               const uint8_t *seen, int64_t seen_stride, int32_t *accept_len,
+                               int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * ts_accept_greedy for callers that have no device memory to give and cannot get any.  (The paper

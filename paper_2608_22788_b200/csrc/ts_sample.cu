@@ -24,6 +24,7 @@ constexpr int kMaxTopK = 32;
 constexpr int kMaxChunks = 16;
 constexpr int kCap = 2048;                                   // candidate slots per chunk
 
+// 16-bit ordered key of a bf16 value (thresholds only): NaN -> 0, -0 = +0, larger value -> larger key.
 __device__ __forceinline__ uint32_t bf16_key(uint32_t u)
 {
     u &= 0xffffu;
@@ -37,6 +38,44 @@ __device__ __forceinline__ uint32_t key_to_bf16(uint32_t key)
 {
     const uint32_t ord = key - 1u;
     return (ord & 0x8000u) ? (ord & 0x7fffu) : (~ord & 0xffffu);
+}
+// 32-bit ordered key of an fp32 value (candidates: a penalised logit is no bf16 number any more).
+__device__ __forceinline__ uint32_t f32_key(uint32_t f)
+{
+    if ((f & 0x7fffffffu) > 0x7f800000u) return 0u;  // NaN
+    if (f == 0x80000000u) f = 0u;                      // -0 -> +0
+    const uint32_t ord = (f & 0x80000000u) ? ~f : (f | 0x80000000u);
+    return ord + 1u;
+}
+__device__ __forceinline__ float key_to_f32(uint32_t key)
+{
+    const uint32_t ord = key - 1u;
+    return __uint_as_float((ord & 0x80000000u) ? (ord & 0x7fffffffu) : ~ord);
+}
+// Key of element idx of a row: its bf16 bits as they are, or -- if the token is present -- of the original
+// logit (re-read from memory: the register copy was rounded) minus the penalty, in fp32.
+__device__ __forceinline__ uint32_t element_key(uint32_t bits16, bool present, const uint16_t *rowp, int idx, float pen)
+{
+    if (!present) return f32_key((bits16 & 0xffffu) << 16);
+    const float y = __uint_as_float((uint32_t)rowp[idx] << 16) - pen;
+    return f32_key(__float_as_uint(y));
+}
+// Register copy of a penalised logit: (logit - penalty) rounded DOWN to bf16.  Thresholds and the candidate
+// test work on these copies; rounding down keeps both sound (a bf16 threshold T is <= x iff T <= rd(x)).
+__device__ __forceinline__ uint32_t penalised_rd(uint32_t bits16, float pen)
+{
+    const float y = __uint_as_float((bits16 & 0xffffu) << 16) - pen;
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(y));
+}
+__device__ __forceinline__ void patch_vector(uint4 &x, uint32_t m, float pen)
+{
+    uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (m & (1u << (2 * i))) w[i] = (w[i] & 0xffff0000u) | penalised_rd(w[i], pen);
+        if (m & (2u << (2 * i))) w[i] = (w[i] & 0x0000ffffu) | (penalised_rd(w[i] >> 16, pen) << 16);
+    }
+    x = make_uint4(w[0], w[1], w[2], w[3]);
 }
 __device__ __forceinline__ uint4 ld_stream_16B(const void *p)
 {
@@ -52,21 +91,45 @@ __device__ __forceinline__ unsigned long long pack_key(uint32_t key16, int idx)
 }
 
 __device__ __noinline__ void push_candidates(uint4 v, uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, int idx0,
-                                             int *cnt, unsigned long long *cand)
+                                             int *cnt, unsigned long long *cand, uint32_t present, const uint16_t *rowp,
+                                             float pen)
 {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     const uint32_t e[4] = {e0, e1, e2, e3};
     for (int i = 0; i < 4; ++i) {
-        if (e[i] & 0xffffu) { const int s = atomicAdd(cnt, 1); if (s < kCap) cand[s] = pack_key(bf16_key(w[i]), idx0 + 2 * i); }
-        if (e[i] >> 16) { const int s = atomicAdd(cnt, 1); if (s < kCap) cand[s] = pack_key(bf16_key(w[i] >> 16), idx0 + 2 * i + 1); }
+        if (e[i] & 0xffffu) {
+            const int s = atomicAdd(cnt, 1);
+            if (s < kCap) cand[s] = pack_key(element_key(w[i], (present >> (2 * i)) & 1u, rowp, idx0 + 2 * i, pen), idx0 + 2 * i);
+        }
+        if (e[i] >> 16) {
+            const int s = atomicAdd(cnt, 1);
+            if (s < kCap)
+                cand[s] = pack_key(element_key(w[i] >> 16, (present >> (2 * i + 1)) & 1u, rowp, idx0 + 2 * i + 1, pen), idx0 + 2 * i + 1);
+        }
     }
 }
 
 // Degenerate chunk (thousands of ties at the threshold): extract the best key below the previous
 // one, top_k times, re-reading the chunk from memory each time.  Slow, exact, and only reached by
 // pathological inputs such as a constant row.
+// The tokens of a chunk that are present for its row, beyond the caller's bitmap: the block's earlier
+// drafts that fall into the chunk, as (vector index, bit of the element inside the vector) pairs.
+struct DraftHits {
+    int n;
+    int vec[256];
+    uint8_t bit[256];
+};
+__device__ __forceinline__ uint32_t present_mask(int j, const uint8_t *srow, const DraftHits *dh)
+{
+    uint32_t m = srow ? srow[j] : 0u;
+    for (int e = 0; e < dh->n; ++e)
+        if (dh->vec[e] == j) m |= dh->bit[e];
+    return m;
+}
+
 __device__ __noinline__ void slow_topk(const uint4 *base, int nvec, int begin, int top_k, unsigned long long *dst,
-                                       unsigned long long *s_red)
+                                       unsigned long long *s_red, const uint8_t *srow, const DraftHits *dh,
+                                       const uint16_t *rowp, float pen)
 {
     const int tid = threadIdx.x;
     unsigned long long prev = ~0ull;
@@ -76,9 +139,11 @@ __device__ __noinline__ void slow_topk(const uint4 *base, int nvec, int begin, i
             const uint4 x = base[j];
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
             const int idx0 = begin + j * 8;
+            const uint32_t pm = pen != 0.f ? present_mask(j, srow, dh) : 0u;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t ka = bf16_key(w[i]), kb = bf16_key(w[i] >> 16);
+                const uint32_t ka = element_key(w[i], (pm >> (2 * i)) & 1u, rowp, idx0 + 2 * i, pen);
+                const uint32_t kb = element_key(w[i] >> 16, (pm >> (2 * i + 1)) & 1u, rowp, idx0 + 2 * i + 1, pen);
                 const unsigned long long a = pack_key(ka, idx0 + 2 * i), b = pack_key(kb, idx0 + 2 * i + 1);
                 if (ka && a < prev && a > best) best = a;
                 if (kb && b < prev && b > best) best = b;
@@ -99,10 +164,14 @@ __device__ __noinline__ void slow_topk(const uint4 *base, int nvec, int begin, i
 }
 
 // grid = (chunks, rows).  out[(row * chunks + chunk) * top_k + j] = j-th best key of the chunk (0 = none).
+// PEN: a presence penalty applies (seen-token bitmap and / or earlier drafts of the block).
+template <bool PEN>
 __global__ void __launch_bounds__(kThreads, 3)
 ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len, int top_k,
-                     unsigned long long *__restrict__ out)
+                     unsigned long long *__restrict__ out, const uint8_t *__restrict__ seen, long long seen_stride,
+                     float pen, const int32_t *__restrict__ draft, int gamma)
 {
+    __shared__ DraftHits s_dh;
     __shared__ unsigned long long s_cand[kCap];
     __shared__ unsigned long long s_red[kThreads / 32];
     __shared__ int s_cnt;
@@ -114,7 +183,8 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
     int end = begin + chunk_len;
     if (end > vocab) end = vocab;
     const int nvec = end > begin ? (end - begin) >> 3 : 0;
-    const uint4 *base = reinterpret_cast<const uint4 *>(logits + (long long)row * row_stride + begin);
+    const uint16_t *rowp = logits + (long long)row * row_stride;
+    const uint4 *base = reinterpret_cast<const uint4 *>(rowp + begin);
     unsigned long long *dst = out + ((long long)row * chunks + chunk) * top_k;
     const uint32_t nan2 = 0x7fc07fc0u;
     uint4 v[kVecPerThread];
@@ -123,7 +193,45 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
         const int j = tid + u * kThreads;
         v[u] = j < nvec ? ld_stream_16B(base + j) : make_uint4(nan2, nan2, nan2, nan2);
     }
-    if (tid == 0) s_cnt = 0;
+    if (tid == 0) { s_cnt = 0; s_dh.n = 0; }
+    // ---- presence penalty: lower the register copies of the present tokens (rounded down to bf16)
+    uint32_t pmask[kVecPerThread / 4];                  // one byte per vector: which of its 8 elements are present
+    const uint8_t *srow = nullptr;
+    if (PEN) {
+        const int R = gamma + 1, b = row / R, irow = row % R;
+        srow = seen ? seen + (long long)b * seen_stride + (begin >> 3) : nullptr;
+        __syncthreads();
+        for (int jj = tid; jj < irow; jj += kThreads) {
+            const int d = draft[(long long)b * gamma + jj];
+            if (d >= begin && d < end) {
+                const int slot = atomicAdd(&s_dh.n, 1);
+                s_dh.vec[slot] = (d - begin) >> 3;
+                s_dh.bit[slot] = (uint8_t)(1u << (d & 7));
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kVecPerThread / 4; ++q) pmask[q] = 0u;
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int j = tid + u * kThreads;
+            if (srow && j < nvec) pmask[u >> 2] |= (uint32_t)srow[j] << (8 * (u & 3));
+        }
+        for (int e = 0; e < s_dh.n; ++e) {
+            const int j = s_dh.vec[e];
+            if ((j & (kThreads - 1)) == tid) {
+                const int u = j >> 8;
+#pragma unroll
+                for (int q = 0; q < kVecPerThread / 4; ++q)
+                    if (q == (u >> 2)) pmask[q] |= (uint32_t)s_dh.bit[e] << (8 * (u & 3));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const uint32_t m = (pmask[u >> 2] >> (8 * (u & 3))) & 0xffu;
+            if (m) patch_vector(v[u], m, pen);
+        }
+    }
     // ---- the largest element of every thread (NaN never wins)
     __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162 *>(&nan2);
 #pragma unroll
@@ -170,7 +278,9 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
         const uint32_t e1 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].y), tt);
         const uint32_t e2 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].z), tt);
         const uint32_t e3 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&v[u].w), tt);
-        if (e0 | e1 | e2 | e3) push_candidates(v[u], e0, e1, e2, e3, begin + (tid + u * kThreads) * 8, &s_cnt, s_cand);
+        if (e0 | e1 | e2 | e3)
+            push_candidates(v[u], e0, e1, e2, e3, begin + (tid + u * kThreads) * 8, &s_cnt, s_cand,
+                            PEN ? (pmask[u >> 2] >> (8 * (u & 3))) & 0xffu : 0u, rowp, pen);
     }
     for (int j = tid; j < top_k; j += kThreads) dst[j] = 0ull;
     __syncthreads();
@@ -184,7 +294,7 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
             if (rank < top_k) dst[rank] = mine;
         }
     } else {
-        slow_topk(base, nvec, begin, top_k, dst, s_red);
+        slow_topk(base, nvec, begin, top_k, dst, s_red, srow, &s_dh, rowp, PEN ? pen : 0.f);
     }
 }
 
@@ -192,7 +302,7 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
 // then walks the draft block with one kept token per lane.
 __global__ void __launch_bounds__(1024)
 ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks, int top_k,
-                        const uint16_t *__restrict__ logits, long long row_stride, const int32_t *__restrict__ draft,
+                        const int32_t *__restrict__ draft,
                         const float *__restrict__ uniforms, int gamma, float inv_temperature, float top_p,
                         int32_t *accept_len, int32_t *out_tokens)
 {
@@ -226,9 +336,9 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         const unsigned long long key = best[lane];
         const bool valid = lane < top_k && key != 0ull;
         const int idx = valid ? (int)(0xffffffffu - (uint32_t)(key & 0xffffffffull)) : -1;
-        // the logit itself (bf16 -> fp32, exact)
+        // the (penalised) logit itself, carried exactly by the key
         float x = -INFINITY;
-        if (valid) x = __uint_as_float((uint32_t)logits[row * row_stride + idx] << 16);
+        if (valid) x = key_to_f32((uint32_t)(key >> 32));
         const float z = x * inv_temperature;
         const float z0 = __shfl_sync(FULL, z, 0);
         float e = valid ? expf(z - z0) : 0.f;
@@ -324,7 +434,19 @@ int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draf
                      int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k, float top_p,
                      int32_t *accept_len, int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream)
 {
+    return ts_accept_sample_penalized(logits, row_stride, draft, uniforms, num_seqs, gamma, vocab, temperature, top_k,
+                                      top_p, 0.f, nullptr, 0, accept_len, out_tokens, workspace, workspace_bytes, stream);
+}
+
+int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int32_t *draft, const float *uniforms,
+                               int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k,
+                               float top_p, float presence_penalty, const uint8_t *seen, int64_t seen_stride,
+                               int32_t *accept_len, int32_t *out_tokens, void *workspace, size_t workspace_bytes,
+                               void *stream)
+{
     using namespace ts::smp;
+    if (isnan(presence_penalty) || isinf(presence_penalty)) return TS_ERR_INVALID_ARG;
+    if (seen && seen_stride * 8 < vocab) return TS_ERR_INVALID_ARG;
     if (num_seqs < 0 || gamma < 0 || vocab < 1) return TS_ERR_INVALID_ARG;
     if (!logits || !uniforms || !accept_len || !out_tokens || !workspace) return TS_ERR_INVALID_ARG;
     if (gamma > 0 && !draft) return TS_ERR_INVALID_ARG;
@@ -346,8 +468,15 @@ int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draf
     chunk_len = (chunk_len + 7) / 8 * 8;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned long long *keys = static_cast<unsigned long long *>(workspace);
-    ts_topk_chunk_kernel<<<dim3((unsigned)chunks, (unsigned)rows), kThreads, 0, s>>>(
-        static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, top_k, keys);
+    // a penalty of zero, or nothing present (no bitmap and no earlier drafts), is the plain kernel
+    if (presence_penalty != 0.f && (seen || gamma > 0))
+        ts_topk_chunk_kernel<true><<<dim3((unsigned)chunks, (unsigned)rows), kThreads, 0, s>>>(
+            static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, top_k, keys, seen, seen_stride,
+            presence_penalty, draft, gamma);
+    else
+        ts_topk_chunk_kernel<false><<<dim3((unsigned)chunks, (unsigned)rows), kThreads, 0, s>>>(
+            static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, top_k, keys, nullptr, 0, 0.f, draft,
+            gamma);
     if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
     const int R = gamma + 1;
     int warps = R < 32 ? R : 32;
@@ -361,8 +490,7 @@ int ts_accept_sample(const void *logits, int64_t row_stride, const int32_t *draf
     const char *pdl = getenv("TS_PDL");
     const bool overlap = !(pdl && pdl[0] == '0');
     const cudaError_t e = ts::launch_overlapped(ts_sample_finish_kernel, dim3((unsigned)num_seqs), dim3(warps * 32), smem, s,
-                                                overlap, (const unsigned long long *)keys, chunks, (int)top_k,
-                                                static_cast<const uint16_t *>(logits), (long long)row_stride, draft,
+                                                overlap, (const unsigned long long *)keys, chunks, (int)top_k, draft,
                                                 uniforms, (int)gamma, 1.0f / temperature, top_p, accept_len, out_tokens);
     return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 MARGIN = 1e-5
 
 
-def run_gpu(logits_bits, draft, u32, T, k, pnuc):
+def run_gpu(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0):
     B, R, V = logits_bits.shape
     gamma = R - 1
     lg = torch.from_numpy(np.ascontiguousarray(logits_bits).view(np.int16)).cuda().view(torch.bfloat16)
@@ -26,7 +26,8 @@ def run_gpu(logits_bits, draft, u32, T, k, pnuc):
     acc = torch.full((B,), -5, dtype=torch.int32, device="cuda")
     out = torch.full((B, R), -5, dtype=torch.int32, device="cuda")
     ws = torch.empty(api.sample_workspace_bytes(B, gamma, V, k), dtype=torch.uint8, device="cuda")
-    api.ts_accept_sample(lg, dr, uu, acc, out, ws, temperature=T, top_k=k, top_p=pnuc)
+    sd = torch.from_numpy(np.ascontiguousarray(seen)).cuda() if seen is not None else None
+    api.ts_accept_sample(lg, dr, uu, acc, out, ws, temperature=T, top_k=k, top_p=pnuc, presence_penalty=pen, seen=sd)
     torch.cuda.synchronize()
     return acc.cpu().numpy(), out.cpu().numpy()
 
@@ -53,12 +54,13 @@ def near_tie(b, i, draft, u, ids, pp, gamma, pnuc):
     return False
 
 
-def check(logits_bits, draft, u32, T, k, pnuc):
+def check(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0):
     B, R, V = logits_bits.shape
     gamma = R - 1
     u = np.asarray(u32, np.float32)
-    racc, rout, ids, pp = oracle.accept_sample(logits_bits, draft, u.astype(np.float64), temperature=T, top_k=k, top_p=pnuc)
-    gacc, gout = run_gpu(logits_bits, draft, u, T, k, pnuc)
+    racc, rout, ids, pp = oracle.accept_sample(logits_bits, draft, u.astype(np.float64), temperature=T, top_k=k, top_p=pnuc,
+                                               seen=seen, presence_penalty=pen)
+    gacc, gout = run_gpu(logits_bits, draft, u, T, k, pnuc, seen, pen)
     undecided = 0
     for b in range(B):
         if gacc[b] == racc[b] and np.array_equal(gout[b], rout[b]):
@@ -134,3 +136,85 @@ def test_argument_errors():
                     (dict(temperature=0.7, top_k=20, top_p=0.0), "TS_ERR_INVALID_ARG")):
         with pytest.raises(api.TailSieveError, match=err):
             api.ts_accept_sample(lg, None, u, acc, out, ws, **kw)
+
+
+# ------------------------------------------------------------------------------------------------
+# presence penalty
+# ------------------------------------------------------------------------------------------------
+def _bitmap(B, V, rng, density, stride=None):
+    nbytes = (V + 7) // 8
+    stride = stride or nbytes
+    bm = np.zeros((B, stride), np.uint8)
+    bits = rng.random((B, V)) < density
+    bm[:, :nbytes] = np.packbits(bits, axis=1, bitorder="little")[:, :nbytes]
+    return bm
+
+
+@pytest.mark.parametrize("gamma,density", [(0, 0.1), (4, 0.1), (16, 0.02), (8, 0.5)])
+def test_presence_penalty_paper_regime_full_vocab(gamma, density):
+    # the paper's sampling table: temperature 0.7, top-k 20, top-p 0.8, presence penalty 1.5
+    B, V = 16, wl.VOCAB
+    rng = np.random.default_rng(50 + gamma)
+    logits = wl.make_logits(B, gamma, V, seed=60 + gamma)
+    f = wl.bf16_bits_to_f32(logits)
+    best = np.argmax(f, -1)
+    draft = np.where(rng.random((B, gamma)) < 0.8, best[:, :gamma], rng.integers(0, V, (B, gamma))).astype(np.int32)
+    if gamma >= 2:
+        draft[0, 1] = draft[0, 0]                    # a repeated draft: row 2 of sequence 0 sees it once
+    seen = _bitmap(B, V, rng, density, stride=(V + 7) // 8 + 16)
+    # make sure the penalty matters: the best tokens of half of the rows are marked as seen
+    for b in range(0, B, 2):
+        for v in best[b]:
+            seen[b, v >> 3] |= np.uint8(1 << (v & 7))
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    acc, out = check(logits, draft, u, 0.7, 20, 0.8, seen=seen, pen=1.5)
+    plain_acc, plain_out, _, _ = oracle.accept_sample(logits, draft, u.astype(np.float64), temperature=0.7, top_k=20, top_p=0.8)
+    assert not (np.array_equal(acc, plain_acc) and np.array_equal(out, plain_out))     # the penalty changed something
+
+
+def test_presence_penalty_without_bitmap_counts_the_earlier_drafts():
+    B, gamma, V = 24, 6, 8192
+    rng = np.random.default_rng(77)
+    logits = wl.make_logits(B, gamma, V, seed=78)
+    best = np.argmax(wl.bf16_bits_to_f32(logits), -1)
+    draft = best[:, :gamma].astype(np.int32).copy()
+    draft[:, 1:] = draft[:, :1]                      # the same token drafted again and again
+    logits[:, :, :] = logits[:, :1, :]               # and the same distribution at every position
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    check(logits, draft, u, 0.7, 20, 0.8, seen=None, pen=4.0)
+
+
+def test_presence_penalty_ties_negative_penalty_and_slow_path():
+    # constant rows (thousands of ties, the exact fallback path) with a few seen tokens, a negative penalty
+    # (a bonus: seen tokens move up), and -inf / NaN logits that a penalty must leave alone
+    B, gamma, V = 6, 2, 40000
+    rng = np.random.default_rng(5)
+    base = np.zeros((B, gamma + 1, V), np.float32)
+    base[1] = -3.0
+    base[2, :, ::2] = -np.inf
+    base[3, :, 5] = np.nan
+    base[4] = rng.integers(-4, 5, (gamma + 1, V)).astype(np.float32)
+    base[5] = 1.0
+    logits = wl.f32_to_bf16_bits(base)
+    seen = _bitmap(B, V, rng, 0.001)
+    for b in range(B):
+        for v in (0, 1, 5, 9, V - 1):
+            seen[b, v >> 3] |= np.uint8(1 << (v & 7))
+    draft = rng.integers(0, 16, (B, gamma)).astype(np.int32)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    check(logits, draft, u, 0.7, 20, 0.8, seen=seen, pen=1.5)
+    check(logits, draft, u, 1.0, 8, 1.0, seen=seen, pen=-2.25)
+
+
+def test_presence_penalty_argument_errors():
+    B, V = 2, 4096
+    lg = torch.zeros((B, 1, V), dtype=torch.bfloat16, device="cuda")
+    u = torch.zeros((B, 1, 2), dtype=torch.float32, device="cuda")
+    acc = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    out = torch.zeros((B, 1), dtype=torch.int32, device="cuda")
+    ws = torch.empty(api.sample_workspace_bytes(B, 0, V, 20), dtype=torch.uint8, device="cuda")
+    short = torch.zeros((B, V // 8 - 1), dtype=torch.uint8, device="cuda")
+    with pytest.raises(api.TailSieveError):
+        api.ts_accept_sample(lg, None, u, acc, out, ws, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=1.5, seen=short)
+    with pytest.raises(api.TailSieveError):
+        api.ts_accept_sample(lg, None, u, acc, out, ws, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=float("nan"))
