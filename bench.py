@@ -406,6 +406,8 @@ def run_ours(args):
     extras = {}
     if not args.headline_only:
         extras = run_extras(torch, api, W, pool, peak, seed, quick=args.quick)
+        del W
+        extras["variants:attention"] = run_variants(torch, api, peak, seed)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
@@ -652,6 +654,55 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         out["mixed:split_into_bulk_and_tail_calls"] = {"bulk_ms": mb, "tail_ms": mt, "sum_ms": mb + mt,
                                                        "uniform_ms": out["mixed:ts_decode_attn"]["ms"],
                                                        "tail_seqs": int(len(wt_lens))}
+    return out
+
+
+def run_variants(torch, api, peak, seed):
+    """Decode and verify attention on the bulk and tail lengths with other geometries (page sizes, pool
+    layout, query heads per kv head, kv heads per GPU, head_dim 64).  Pools are filled on the device with
+    seeded normal values (only their size and layout matter for timing)."""
+    flush = L2Flusher()
+    out = {}
+    gen = torch.Generator(device="cuda")
+
+    def one(tag, lens, D, P, Hkv, Hq, q_len, layout):
+        lens = np.asarray(lens, dtype=np.int32)
+        B = len(lens)
+        npg = (lens + P - 1) // P
+        total = int(npg.sum())
+        pages = total + 64
+        perm = np.random.default_rng([seed, 91]).permutation(pages)[:total].astype(np.int32)
+        mp = int(npg.max())
+        bt = np.zeros((B, mp), dtype=np.int32)
+        o = 0
+        for s_ in range(B):
+            bt[s_, :npg[s_]] = perm[o:o + npg[s_]]
+            o += npg[s_]
+        if layout == "HND":
+            shape, ps, ts_, hs = (pages, Hkv, P, D), Hkv * P * D, D, P * D
+        else:
+            shape, ps, ts_, hs = (pages, P, Hkv, D), Hkv * P * D, Hkv * D, D
+        gen.manual_seed(seed * 7919 + 13)
+        k = torch.randn(shape, device="cuda", dtype=torch.bfloat16, generator=gen)
+        v = torch.randn(shape, device="cuda", dtype=torch.bfloat16, generator=gen)
+        q = torch.randn((B, q_len, Hq, D), device="cuda", dtype=torch.bfloat16, generator=gen)
+        o_ = torch.empty_like(q)
+        geom = api.AttnGeometry(B, q_len, Hq, Hkv, D, P, pages, mp, ps, ts_, hs, 1.0 / float(np.sqrt(D)))
+        ws = torch.empty(api.attn_workspace_bytes(geom), dtype=torch.uint8, device="cuda")
+        btd, ld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
+        f = api.ts_verify_attn if q_len > 1 else api.ts_decode_attn
+        med, mn = time_with_flush(lambda: f(geom, q, k, v, btd, ld, o_, ws), flush, iters=5, warmup=2)
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        nbytes = int(lens.sum()) * Hkv * D * 4 + 2 * B * q_len * Hq * D * 2
+        out[tag] = {"ms": med, "GBps": gbs(nbytes, med), "frac_of_measured_peak": gbs(nbytes, med) / peak,
+                    "algorithmic_bytes": nbytes}
+        del k, v, q, o_
+
+    for name, lens in (("bulk", wl.lens_bulk(seed)), ("tail", wl.lens_tail(seed))):
+        for (D, P, Hkv, Hq, ql, lay) in ((128, 16, 8, 32, 1, "HND"), (128, 32, 8, 32, 1, "HND"), (128, 128, 8, 32, 1, "HND"),
+                                         (128, 64, 8, 32, 1, "NHD"), (128, 64, 8, 8, 1, "HND"), (128, 64, 8, 64, 1, "HND"),
+                                         (128, 64, 4, 16, 1, "HND"), (64, 64, 8, 32, 1, "HND"), (128, 64, 8, 64, 5, "HND")):
+            one(f"{name}:D{D}_P{P}_{lay}_Hq{Hq}_Hkv{Hkv}_q{ql}", lens, D, P, Hkv, Hq, ql, lay)
     return out
 
 
