@@ -422,14 +422,24 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     } else {
         // ============================================================ softmax warpgroups (one thread per row)
         const int wg = (warp - 3) >> 2;                   // 0 or 1: parity of the tiles this group takes
+        // A warp reaches the 32 TMEM lanes of its quarter q4 = warp % 4 only, and warp % 4 is also the SM
+        // sub-partition (scheduler) it issues from.  Sub-partition 3 hosts no single-thread role, 0 the TMA
+        // producer, 2 the PV issuer, 1 the QK issuer, so the 32-row blocks of a pair are handed to the
+        // quarters in that order: with few rows the busy softmax warps stay off the MMA issuers' schedulers.
         const int q4 = warp & 3;
-        const int row = q4 * 32 + lane;
+        const int blk = (0x0231 >> (4 * q4)) & 3;         // quarter 3 -> rows 0..31, 0 -> 32..63, 2 -> 64..95, 1 -> 96..127
+        const int mrow = q4 * 32 + lane;                  // row of the MMA tile = TMEM lane = row of the Q tile
+        const int row = blk * 32 + lane;                  // query row of the pair that lives there
         const uint32_t tlane = (uint32_t)(q4 * 32) << 16;
         const bool row_valid = row < a.rows;
         const int t_row = row_valid ? row / a.G : 0, hl = row_valid ? row % a.G : 0;
         const int tid_wg = (threadIdx.x - 96) & 127;      // 0..127 inside the group
+        // A warp none of whose 32 rows exists has nothing to compute: its rows of Q are zeros, so its rows of
+        // S are zeros (or NaN under a poisoned key), which is all the P those rows need -- nobody reads their
+        // O.  It only keeps step with the barriers.  At 20 rows (gamma 4) that is 3 of a group's 4 warps.
+        const bool idle_warp = blk * 32 >= a.rows;
         const uint32_t o_col = kTmemO + (uint32_t)wg * 128u;
-        const uint32_t stats = base + kOffStats + (uint32_t)row * 8u;
+        const uint32_t stats = base + kOffStats + (uint32_t)mrow * 8u;
         // This group's PVs are numbered u = it >> 1; PV u signals pdone of buffer 2*wg + (u & 1), phase u >> 1.
         // A parity wait only tells the current phase from the previous one, so the phases of each of the two
         // barriers are observed in order, and PV u - 2 (the previous phase of the barrier PV u will signal) is
@@ -447,11 +457,11 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         // zero-filled): this thread's row, as asynchronous 16-byte copies.
         auto issue_q = [&](int s_, int g_) {
             const uint16_t *src = a.q + (((size_t)s_ * a.q_len + t_row) * a.Hq + (size_t)g_ * a.G + hl) * D;
-            const uint32_t qrow = base + kOffQ + (uint32_t)row * 128u;
+            const uint32_t qrow = base + kOffQ + (uint32_t)mrow * 128u;
             const uint32_t nbytes = row_valid ? 16u : 0u;
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
-                const uint32_t addr = qrow + (uint32_t)(c >> 3) * 16384u + (uint32_t)(((c & 7) ^ (row & 7)) << 4);
+                const uint32_t addr = qrow + (uint32_t)(c >> 3) * 16384u + (uint32_t)(((c & 7) ^ (mrow & 7)) << 4);
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(addr), "l"(src + 8 * c), "r"(nbytes) : "memory");
             }
         };
@@ -502,6 +512,10 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 wait(sfull(buf), (uint32_t)(it >> 2) & 1u);
                 fence_after_sync();
                 TS_TRACE(1)
+                float alpha = 1.f, rowsum = 0.f;
+                bool rescale = false;
+                const bool need_mask = tok0 + kTile - 1 > sg.n - a.q_len;
+                if (!idle_warp) {
                 uint32_t xr[2][32];
                 tmem_ld32(sp_tmem, xr[0]);
                 tmem_ld32(sp_tmem + 32, xr[1]);
@@ -509,7 +523,6 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 TS_TRACE(2)
                 if (q4 == 3 && lane == 0) TS_EVENT(it, 3)
                 // mask (only near the sequence end) and row maximum of the raw scores (scale > 0 here)
-                const bool need_mask = tok0 + kTile - 1 > sg.n - a.q_len;
                 if (need_mask) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
@@ -524,8 +537,6 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(xr[h][c]));
                 const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
                 const float m_new = fmaxf(m_used, mx);
-                float alpha = 1.f;
-                bool rescale = false;
                 if (j < 2 || m_new > m_used + kLazyTau) {
                     alpha = ex2(m_used - ((m_new == -INFINITY) ? 0.f : m_new));
                     rescale = (j >= 2) && (m_new != m_used);
@@ -549,7 +560,8 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     tmem_st16(sp_tmem + 16 * h, hi);
                     tmem_st16(sp_tmem + 32 + 16 * h, lo);
                 }
-                const float rowsum = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                rowsum = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                }
                 TS_TRACE(4)
                 // V rows past the sequence end may hold anything: zero them (0 * NaN)
                 const int valid_tok = sg.n - tok0;
@@ -563,7 +575,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     }
                 }
                 const int u = it >> 1;
-                if (u >= 2) observe_upto(u - 2);
+                if (u >= 2 && !idle_warp) observe_upto(u - 2);
                 // lazy rescale of this group's O in TMEM (warp-collective): every PV into it must have finished
                 if (__any_sync(FULL, rescale)) {
                     observe_upto(u - 1);
@@ -590,7 +602,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 TS_TRACE(5)
             }
             // ---- end of the segment: merge the two groups' accumulators, write the result
-            if (last_t >= 0) observe_upto(last_t >> 1);
+            if (last_t >= 0 && !idle_warp) observe_upto(last_t >> 1);
             if (q4 == 3 && lane == 0) TS_EVENT(it0 + sg.len - 1, 8 + wg)
             if (need_o_sync) named_bar_sync(3, 256);      // no tile of this segment was ours: still pair up
             if (wg == 1) {
