@@ -188,6 +188,10 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = blockIdx.x;
+    // Up to 64 rows per pair the MMAs are issued with M = 64: half of the tensor datapath stays idle, which
+    // is what the sustained speed of this power-bound kernel turns on.  An M = 64 tile keeps row 16 j + i
+    // (i < 16) in TMEM lane 32 j + i, accumulators and the P operand alike.
+    const bool m64 = a.rows <= 64;
 
     // barrier addresses
     const uint32_t bar0 = base + kOffBar;
@@ -324,7 +328,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     } else if (warp == 1) {
         // ============================================================ first MMA issuer: S = Q . K^T
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0);
+            const uint32_t idesc_qk = m64 ? idesc_bf16(64, 64, 0) : idesc_bf16(128, 64, 0);
             const uint64_t dk = smem_desc_sw128(0, 16, 1024);          // K-major operands (Q, K tile)
             const uint32_t q_lo = ((base + kOffQ) & 0x3ffffu) >> 4;
             int t = 0, remaining = total, seg_no = 0, st = 0;
@@ -373,7 +377,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     } else if (warp == 2) {
         // ============================================================ second MMA issuer: O += P . V
         if (lane == 0) {
-            constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 1);
+            const uint32_t idesc_pv = m64 ? idesc_bf16(64, 128, 1) : idesc_bf16(128, 128, 1);
             const uint64_t dv = smem_desc_sw128(0, 8192, 1024);        // MN-major operand (V tile)
             int t = 0, remaining = total, st = 0;
             uint32_t st_par = 0;
@@ -427,17 +431,21 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         // producer, 2 the PV issuer, 1 the QK issuer, so the 32-row blocks of a pair are handed to the
         // quarters in that order: with few rows the busy softmax warps stay off the MMA issuers' schedulers.
         const int q4 = warp & 3;
-        const int blk = (0x0231 >> (4 * q4)) & 3;         // quarter 3 -> rows 0..31, 0 -> 32..63, 2 -> 64..95, 1 -> 96..127
-        const int mrow = q4 * 32 + lane;                  // row of the MMA tile = TMEM lane = row of the Q tile
-        const int row = blk * 32 + lane;                  // query row of the pair that lives there
+        const int blk = (0x0231 >> (4 * q4)) & 3;         // quarter 3 -> first block of rows, then 0, 2, 1
+        const int per_q = m64 ? 16 : 32;                  // rows of the MMA tile per quarter
+        const bool lane_used = lane < per_q;
+        // row of the MMA tile (= row of the Q tile in shared memory) behind this thread's TMEM lane; the
+        // unused upper lanes of an M = 64 quarter get indices past the tile (scratch slots, never a tile row)
+        const int mrow = lane_used ? q4 * per_q + lane : 64 + q4 * 16 + (lane - 16);
+        const int row = blk * per_q + lane;               // query row of the pair that lives there
         const uint32_t tlane = (uint32_t)(q4 * 32) << 16;
-        const bool row_valid = row < a.rows;
+        const bool row_valid = lane_used && row < a.rows;
         const int t_row = row_valid ? row / a.G : 0, hl = row_valid ? row % a.G : 0;
         const int tid_wg = (threadIdx.x - 96) & 127;      // 0..127 inside the group
         // A warp none of whose 32 rows exists has nothing to compute: its rows of Q are zeros, so its rows of
         // S are zeros (or NaN under a poisoned key), which is all the P those rows need -- nobody reads their
         // O.  It only keeps step with the barriers.  At 20 rows (gamma 4) that is 3 of a group's 4 warps.
-        const bool idle_warp = blk * 32 >= a.rows;
+        const bool idle_warp = blk * per_q >= a.rows;
         const uint32_t o_col = kTmemO + (uint32_t)wg * 128u;
         const uint32_t stats = base + kOffStats + (uint32_t)mrow * 8u;
         // This group's PVs are numbered u = it >> 1; PV u signals pdone of buffer 2*wg + (u & 1), phase u >> 1.
@@ -458,6 +466,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         auto issue_q = [&](int s_, int g_) {
             const uint16_t *src = a.q + (((size_t)s_ * a.q_len + t_row) * a.Hq + (size_t)g_ * a.G + hl) * D;
             const uint32_t qrow = base + kOffQ + (uint32_t)mrow * 128u;
+            if (!lane_used) return;                          // M = 64: the upper lanes of a quarter own no tile row
             const uint32_t nbytes = row_valid ? 16u : 0u;
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
@@ -539,7 +548,7 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                 const float m_new = fmaxf(m_used, mx);
                 if (j < 2 || m_new > m_used + kLazyTau) {
                     alpha = ex2(m_used - ((m_new == -INFINITY) ? 0.f : m_new));
-                    rescale = (j >= 2) && (m_new != m_used);
+                    rescale = row_valid && (j >= 2) && (m_new != m_used);
                     m_used = m_new;
                 }
                 const float mref = (m_used == -INFINITY) ? 0.f : m_used;
