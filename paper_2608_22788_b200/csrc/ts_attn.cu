@@ -966,7 +966,8 @@ static int launch_attn_tc(const CUtensorMap &tk, const CUtensorMap &tv, AttnArgs
 
 static bool use_tc_kernel(int D, int rows, float scale_log2)
 {
-    return D == 128 && rows > 16 && rows <= 128 && scale_log2 > 0.f && env_int("TS_ATTN_TC", 1) != 0;
+    return D == 128 && rows >= env_int("TS_ATTN_TC_MIN_ROWS", 17) && rows <= 128 && scale_log2 > 0.f &&
+           env_int("TS_ATTN_TC", 1) != 0;
 }
 
 template <int D>
