@@ -57,6 +57,8 @@ struct AttnArgs {
     int box_tok;                 // warp-MMA kernel: tokens per 4-D TMA box (16/32/64, <= page size); 0 = one 5-D box per tile
     int lg_page;                 // log2(page size)
     int lg_box;                  // log2(box_tok) when box_tok > 0
+    int page_boxes;              // warp-MMA kernel: 1 = 5-D boxes of one 16-token page x both 64-dim halves (page size 16)
+    int blk_stride, half_stride; // shared-memory tile layout: bytes between 16-token blocks / between the 64-dim halves
     float scale_log2;            // scale * log2(e)
     long long wait_cycles;       // bound of every mbarrier wait
 };
@@ -302,6 +304,17 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 mbar_expect_tx(bv, bytes);
             }
             __syncwarp();
+            if (a.page_boxes) {
+                // 16-token pages: lanes 0..7 = (pool, page of the tile); one 5-D box carries both halves of a
+                // page, landing as [page][half][16 tokens][128 B]
+                const int is_v = lane >> 2, b = lane & 3;
+                if (lane < 8 && b < nbox) {
+                    const int id = b == 0 ? ids[0] : (b == 1 ? ids[1] : (b == 2 ? ids[2] : ids[3]));
+                    tma_load_5d((is_v ? vdst : kdst) + b * bbytes * HALVES, is_v ? (const void *)&tmV : (const void *)&tmK,
+                                0, 0, 0, ic.g, id, is_v ? bv : bk);
+                }
+                return;
+            }
             // lanes 0..7 = (pool, half, box parity): each issues boxes b and b + 2 of its pool and half,
             // so a tile of 32-token boxes goes out in one warp instruction
             const int is_v = lane >> 2, h = (lane >> 1) & 1, b0 = lane & 1;
@@ -412,11 +425,11 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #pragma unroll
             for (int kk = 0; kk < KK; ++kk) {
                 const int chunk = 2 * kk + k_chunk_l;
-                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (kTile * 128);
+                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (uint32_t)a.half_stride;
 #pragma unroll
                 for (int mi = 0; mi < 4; ++mi) {
                     uint32_t af[4];
-                    ldsm_x4(af, kbase + mi * 2048 + k_row_off + col);
+                    ldsm_x4(af, kbase + mi * (uint32_t)a.blk_stride + k_row_off + col);
 #pragma unroll
                     for (int j = 0; j < NT; ++j) mma_bf16_16816(sacc[mi][j], af, bq[j][kk][0], bq[j][kk][1]);
                 }
@@ -496,7 +509,7 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 for (int r = valid_tok + (lane >> 3); r < kTile; r += 4)
 #pragma unroll
                     for (int h = 0; h < HALVES; ++h) {
-                        const uint32_t addr = vbase + h * (kTile * 128) + r * 128 + l7 * 16;
+                        const uint32_t addr = vbase + h * (uint32_t)a.half_stride + (r >> 4) * (uint32_t)a.blk_stride + (r & 15) * 128 + l7 * 16;
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                 __syncwarp();
@@ -504,11 +517,11 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #pragma unroll
             for (int md = 0; md < MD; ++md) {
                 const int chunk = 2 * md + v_chunk_l;
-                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (kTile * 128);
+                const uint32_t col = (uint32_t)(((chunk & 7) ^ l7) << 4) + (uint32_t)(chunk >> 3) * (uint32_t)a.half_stride;
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     uint32_t af[4];
-                    ldsm_x4_trans(af, vbase + ks * 2048 + v_row_off + col);
+                    ldsm_x4_trans(af, vbase + ks * (uint32_t)a.blk_stride + v_row_off + col);
 #pragma unroll
                     for (int j = 0; j < NT; ++j) {
                         mma_bf16_16816(acc_o[md][j], af, bph[ks][j][0], bph[ks][j][1]);
@@ -828,12 +841,27 @@ static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) &
 
 // box_tok = 0: one 5-D box per 64-token tile when the page holds a whole tile, else one 4-D box per page;
 // box_tok > 0: 4-D boxes of that many tokens (must divide 64 and not exceed the page size).
-static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_params *p, int *tok_first, int box_tok_req)
+static int make_tensor_map(CUtensorMap *tm, const void *pool, const ts_attn_params *p, int *tok_first, int box_tok_req,
+                           bool page_boxes = false)
 {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return TS_ERR_CUDA;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r;
+    if (page_boxes) {
+        // 5-D with a box of one whole short page: (64 dims, page_size tokens, all halves) of one head, landing
+        // in shared memory as [half][token][128 B]
+        *tok_first = 1;
+        const cuuint64_t halves = (cuuint64_t)p->head_dim / 64;
+        cuuint64_t dims[5] = {64, (cuuint64_t)p->page_size, halves, (cuuint64_t)p->num_kv_heads, (cuuint64_t)p->num_pages};
+        cuuint64_t strides[4] = {(cuuint64_t)p->kv_token_stride * 2, 128, (cuuint64_t)p->kv_head_stride * 2,
+                                 (cuuint64_t)p->kv_page_stride * 2};
+        cuuint32_t box[5] = {64, (cuuint32_t)p->page_size, (cuuint32_t)halves, 1, 1};
+        r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(pool), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS ? TS_OK : TS_ERR_UNSUPPORTED;
+    }
     if (p->page_size >= kTile && box_tok_req == 0) {
         // 5-D: (64 dims, token, 64-dim half, head, page).  One box = 64 tokens x all halves, laid out in
         // shared memory as [half][token][128 B]: a whole K or V tile per TMA instruction.
@@ -1033,11 +1061,15 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
         if (box_tok != 0 && box_tok != 16 && box_tok != 32 && box_tok != 64) box_tok = 0;
         if (box_tok > p->page_size || (box_tok == 0 && p->page_size < kTile)) box_tok = p->page_size;
     }
+    // 16-token pages at head_dim 128 (warp-MMA kernel): one box per page carrying both halves -- 8 boxes of
+    // 4 KB per tile instead of 16 of 2 KB (TS_ATTN_PAGE_BOXES=0 keeps the latter)
+    const bool page_boxes = !use_tc_kernel(p->head_dim, rows_all, scale_log2) && p->page_size == 16 &&
+                            p->head_dim == 128 && box_tok == 16 && env_int("TS_ATTN_PAGE_BOXES", 1) != 0;
     CUtensorMap tk, tv;
     int tok_first = 1, tf2 = 1;
-    rc = make_tensor_map(&tk, k_pool, p, &tok_first, box_tok);
+    rc = make_tensor_map(&tk, k_pool, p, &tok_first, box_tok, page_boxes);
     if (rc != TS_OK) return rc;
-    rc = make_tensor_map(&tv, v_pool, p, &tf2, box_tok);
+    rc = make_tensor_map(&tv, v_pool, p, &tf2, box_tok, page_boxes);
     if (rc != TS_OK) return rc;
 
     AttnArgs a;
@@ -1061,6 +1093,9 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     while ((1 << a.lg_page) < p->page_size) ++a.lg_page;
     a.lg_box = 0;
     while ((1 << a.lg_box) < box_tok) ++a.lg_box;
+    a.page_boxes = page_boxes ? 1 : 0;
+    a.blk_stride = page_boxes ? 16 * 128 * (p->head_dim / 64) : 16 * 128;
+    a.half_stride = page_boxes ? 16 * 128 : kTile * 128;
     a.scale_log2 = scale_log2;
     a.wait_cycles = (long long)dev.clock_khz * 2000LL;   // about two seconds of SM clocks
 
