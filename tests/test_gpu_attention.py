@@ -50,6 +50,13 @@ SHAPES = [
     ([900, 33, 2500], 3, 32, 8, 128, 128, "NHD"),             # rows 12, page 128, token-major pool
     ([900, 33, 2500], 9, 8, 2, 128, 16, "HND"),               # rows 36 with 16-token pages (4 boxes per tile)
     ([2, 5000], 4, 8, 1, 128, 64, "HND"),                     # rows 32, a single kv head
+    ([800, 100, 2100], 16, 8, 2, 128, 64, "HND"),             # rows 64: the most an M = 64 tile takes
+    ([800, 100, 2100], 13, 10, 2, 128, 64, "NHD"),            # G = 5, rows 65: the first M = 128 case
+    ([800, 100, 2100], 11, 6, 2, 128, 64, "HND"),             # G = 3, rows 33: three 16-row quarters, one with 1 row
+    ([800, 17, 2100], 7, 14, 2, 128, 32, "HND"),              # G = 7, rows 49
+    ([800, 100, 40], 17, 2, 2, 128, 64, "HND"),               # G = 1, rows 17: the fewest the tcgen05 kernel takes
+    ([300, 2000, 31], 1, 32, 8, 128, 16, "HND"),              # decode over 16-token pages (one box per page)
+    ([300, 2000, 31], 2, 32, 8, 128, 16, "NHD"),              # rows 8 over 16-token pages, token-major pool
 ]
 
 
