@@ -1009,7 +1009,8 @@ static int dispatch_attn(int rows, const CUtensorMap &tk, const CUtensorMap &tv,
         return launch_attn_tc(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 8) return launch_attn<D, 1, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 16) return launch_attn<D, 2, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
-    if (rows <= 24 && env_int("TS_ATTN_W22", 1) == 0) return launch_attn<D, 3, 1>(tk, tv, a, sms, smem_optin, stream, dry, ng);
+    // 17..32 rows: two warps of two n-tiles each share a stage (70 % of the HBM peak on the bulk lengths at
+    // 20 rows against 58 % for one warp of three n-tiles)
     if (rows <= 32) return launch_attn<D, 2, 2>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 48) return launch_attn<D, 3, 2>(tk, tv, a, sms, smem_optin, stream, dry, ng);
     if (rows <= 72) return launch_attn<D, 3, 3>(tk, tv, a, sms, smem_optin, stream, dry, ng);
