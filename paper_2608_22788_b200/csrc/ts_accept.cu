@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kArgmaxThreads)
 ts_argmax_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len,
                        unsigned long long *__restrict__ keys)
 {
+    grid_dependency_wait();
     const int chunk = blockIdx.x, row = blockIdx.y, chunks = gridDim.x;
     const uint16_t *base = logits + (long long)row * row_stride;
     const int begin = chunk * chunk_len;
@@ -126,6 +127,7 @@ __global__ void __launch_bounds__(kArgmaxThreads)
 ts_argmax_reg_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len,
                      unsigned long long *__restrict__ keys)
 {
+    grid_dependency_wait();
     const int chunk = blockIdx.x, row = blockIdx.y, chunks = gridDim.x;
     const int begin = chunk * chunk_len;
     int end = begin + chunk_len;
@@ -239,6 +241,8 @@ static int launch_accept(const void *logits, long long row_stride, const int32_t
 {
     const long long rows = (long long)num_seqs * (gamma + 1);
     int chunks, chunk_len;
+    const char *pdl = getenv("TS_PDL");
+    const bool overlap = !(pdl && pdl[0] == '0');     // programmatic dependent launches (every kernel waits first)
     const int fast_chunks = (vocab + kFastChunk - 1) / kFastChunk;
     const bool fast = (row_stride % 8 == 0) && (vocab % 8 == 0) && fast_chunks <= kMaxChunks;
     if (fast) {
@@ -247,18 +251,17 @@ static int launch_accept(const void *logits, long long row_stride, const int32_t
         if (chunks < fast_chunks) chunks = fast_chunks;
         chunk_len = (vocab + chunks - 1) / chunks;
         chunk_len = (chunk_len + 7) / 8 * 8;
-        ts_argmax_reg_kernel<<<dim3((unsigned)chunks, (unsigned)rows), kArgmaxThreads, 0, s>>>(
-            static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys);
+        if (launch_overlapped(ts_argmax_reg_kernel, dim3((unsigned)chunks, (unsigned)rows), dim3(kArgmaxThreads), 0, s,
+                              overlap, static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys) != cudaSuccess)
+            return TS_ERR_CUDA;
     } else {
         chunks = pick_chunks(rows, vocab);
         chunk_len = (vocab + chunks - 1) / chunks;
         chunk_len = (chunk_len + 7) / 8 * 8;
-        ts_argmax_chunk_kernel<<<dim3((unsigned)chunks, (unsigned)rows), kArgmaxThreads, 0, s>>>(
-            static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys);
+        if (launch_overlapped(ts_argmax_chunk_kernel, dim3((unsigned)chunks, (unsigned)rows), dim3(kArgmaxThreads), 0, s,
+                              overlap, static_cast<const uint16_t *>(logits), row_stride, vocab, chunk_len, keys) != cudaSuccess)
+            return TS_ERR_CUDA;
     }
-    if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
-    const char *pdl = getenv("TS_PDL");
-    const bool overlap = !(pdl && pdl[0] == '0');
     const cudaError_t e = launch_overlapped(ts_accept_finish_kernel, dim3(1), dim3(256), 0, s, overlap,
                                             (const unsigned long long *)keys, chunks, draft, num_seqs, gamma,
                                             target_argmax, accept_len, out_tokens);

@@ -85,6 +85,7 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
 {
     __shared__ int warp_sums[32];
     __shared__ int carry_s;
+    grid_dependency_wait();      // launched ahead of the previous kernel's end: nothing is touched before this
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) { carry_s = 0; *status = TS_OK; cum_tiles[0] = 0; }
     __syncthreads();
@@ -1107,12 +1108,15 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     if (rc != TS_OK) return rc;
 
     const int chunks_per_group = env_int("TS_SPLIT_CHUNKS_PER_GROUP", 16);
-    ts_plan_kernel<<<1, 1024, 0, stream>>>(kv_lens, a.B, a.Hkv, NG, mode, max_splits, chunks_per_group,
-                                           reinterpret_cast<int32_t *>(ws + w.cum_tiles),
-                                           reinterpret_cast<GroupStart *>(ws + w.gstart),
-                                           reinterpret_cast<long long *>(ws + w.gpos), num_splits,
-                                           reinterpret_cast<int32_t *>(ws + w.status), a.part_o, a.part_lse,
-                                           p->q_len * p->num_q_heads, p->head_dim);
+    {
+        const bool overlap = env_int("TS_PDL", 1) != 0;
+        const cudaError_t e = launch_overlapped(
+            ts_plan_kernel, dim3(1), dim3(1024), 0, stream, overlap, kv_lens, a.B, a.Hkv, NG, mode, max_splits,
+            chunks_per_group, reinterpret_cast<int32_t *>(ws + w.cum_tiles), reinterpret_cast<GroupStart *>(ws + w.gstart),
+            reinterpret_cast<long long *>(ws + w.gpos), num_splits, reinterpret_cast<int32_t *>(ws + w.status), a.part_o,
+            a.part_lse, p->q_len * p->num_q_heads, p->head_dim);
+        if (e != cudaSuccess) return TS_ERR_CUDA;
+    }
     if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
 
     if (g_ev_start && g_ev_stop) cudaEventRecord(static_cast<cudaEvent_t>(g_ev_start), stream);
