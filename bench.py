@@ -242,7 +242,7 @@ class L2Flusher:
         self.sink = self.rd.sum()
 
 
-def time_with_flush(fn, flush, iters=7, warmup=3):
+def time_with_flush(fn, flush, iters=20, warmup=5):
     """Median / min milliseconds of ``fn`` with an L2 flush (untimed) before every call."""
     import torch
     for _ in range(warmup):
@@ -624,7 +624,7 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
     for route, lens in (("bulk", wl.lens_bulk(seed)), ("tail", wl.lens_verify(seed))):
         for g in (3, 4, 5):
             dw = Workload(f"{route}_verify_g{g}", lens, pool, q_len=1 + g, seed=seed + 20 + g)
-            med, mn = time_with_flush(dw.attn, flush, iters=5, warmup=2)
+            med, mn = time_with_flush(dw.attn, flush, iters=10, warmup=3)
             assert dw.status() == 0
             depth[f"{route}_g{g}"] = {"ms": med, "positions_per_s": dw.b.num_seqs * (1 + g) / (med * 1e-3),
                                       "GBps": gbs(dw.bytes, med), "frac_of_measured_peak": gbs(dw.bytes, med) / peak}
@@ -642,7 +642,7 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         for dr in range(draws):
             lens = pool_lens if c == 1024 else wl.sweep_subset(pool_lens, c, dr, seed)
             sw = Workload(f"sweep{c}", lens, pool, seed=seed + 100 + dr)
-            med, mn = time_with_flush(sw.attn, flush, iters=5, warmup=2)
+            med, mn = time_with_flush(sw.attn, flush, iters=10, warmup=3)
             rows.append((c / (med * 1e-3), gbs(sw.bytes, med), med, int(lens.sum())))
             del sw
         tps = sorted(r[0] for r in rows)
@@ -714,7 +714,7 @@ def run_variants(torch, api, peak, seed):
         ws = torch.empty(api.attn_workspace_bytes(geom), dtype=torch.uint8, device="cuda")
         btd, ld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
         f = api.ts_verify_attn if q_len > 1 else api.ts_decode_attn
-        med, mn = time_with_flush(lambda: f(geom, q, k, v, btd, ld, o_, ws), flush, iters=5, warmup=2)
+        med, mn = time_with_flush(lambda: f(geom, q, k, v, btd, ld, o_, ws), flush, iters=10, warmup=3)
         assert int(ws[:4].view(torch.int32).item()) == 0
         nbytes = int(lens.sum()) * Hkv * D * 4 + 2 * B * q_len * Hq * D * 2
         out[tag] = {"ms": med, "GBps": gbs(nbytes, med), "frac_of_measured_peak": gbs(nbytes, med) / peak,
