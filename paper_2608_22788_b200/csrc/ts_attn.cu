@@ -703,18 +703,19 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     }
 }
 
-// Caller-visible dense layout: one CTA (4 warps) per output row (s, t, h).  The splits of the row
+// Caller-visible dense layout: one CTA (NW warps) per output row (s, t, h).  The splits of the row
 // are dealt round robin to the warps (lanes across head_dim), four loads in flight per warp; the
-// four partial sums are combined through shared memory.
-template <int D>
-__global__ void __launch_bounds__(128)
+// warps' partial sums are combined through shared memory.  NW = 16 when a row can have many parts
+// (a hundred parts over 4 warps is a chain of seven dependent rounds of loads; over 16 warps two).
+template <int D, int NW>
+__global__ void __launch_bounds__(NW * 32)
 ts_merge_dense_kernel(const float *__restrict__ part_o, const float *__restrict__ part_lse,
                       const int32_t *__restrict__ num_splits, uint16_t *out, int B, int rows_all, int max_splits)
 {
     constexpr int V = D / 32;     // floats per lane
-    __shared__ float s_max[4];
-    __shared__ float s_w[4];
-    __shared__ float s_acc[4][D];
+    __shared__ float s_max[NW];
+    __shared__ float s_w[NW];
+    __shared__ float s_acc[NW][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long row = blockIdx.x;
     const int s = (int)(row / rows_all), r = (int)(row % rows_all);
@@ -726,23 +727,25 @@ ts_merge_dense_kernel(const float *__restrict__ part_o, const float *__restrict_
     const float *pl = part_lse + (size_t)s * max_splits * rows_all + r;
     // maximum of the log-sum-exps
     float M = -INFINITY;
-    for (int i = threadIdx.x; i < S; i += 128) M = fmaxf(M, pl[(size_t)i * l_stride]);
+    for (int i = threadIdx.x; i < S; i += NW * 32) M = fmaxf(M, pl[(size_t)i * l_stride]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     if (lane == 0) s_max[warp] = M;
     __syncthreads();
-    M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+    M = s_max[0];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) M = fmaxf(M, s_max[w]);
     float acc[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = 0.f;
     float Wsum = 0.f;
     if (M != -INFINITY) {
-        for (int i0 = warp; i0 < S; i0 += 16) {
+        for (int i0 = warp; i0 < S; i0 += 4 * NW) {
             float w[4];
             float x[4][V];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i = i0 + 4 * u;
+                const int i = i0 + NW * u;
                 const float lse = i < S ? pl[(size_t)i * l_stride] : -INFINITY;
                 w[u] = lse == -INFINITY ? 0.f : expf(lse - M);
                 const float *p = po + (size_t)(i < S ? i : 0) * o_stride + lane * V;
@@ -762,14 +765,17 @@ ts_merge_dense_kernel(const float *__restrict__ part_o, const float *__restrict_
     for (int v = 0; v < V; ++v) s_acc[warp][lane * V + v] = acc[v];
     __syncthreads();
     if (warp == 0) {
-        const float Wt = (s_w[0] + s_w[1]) + (s_w[2] + s_w[3]);
+        float Wt = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) Wt += s_w[w];
         const float inv = Wt > 0.f ? 1.f / Wt : 0.f;
         uint16_t *o = out + (size_t)row * D + lane * V;
 #pragma unroll
         for (int v = 0; v < V; v += 2) {
             const int d = lane * V + v;
-            const float a0 = (s_acc[0][d] + s_acc[1][d]) + (s_acc[2][d] + s_acc[3][d]);
-            const float a1 = (s_acc[0][d + 1] + s_acc[1][d + 1]) + (s_acc[2][d + 1] + s_acc[3][d + 1]);
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { a0 += s_acc[w][d]; a1 += s_acc[w][d + 1]; }
             *reinterpret_cast<uint32_t *>(o + v) = pack_bf16x2(a0 * inv, a1 * inv);
         }
     }
@@ -1202,12 +1208,15 @@ int ts_lse_merge(const ts_attn_params *p, int32_t max_splits, const float *parti
     if (rows > 0x7fffffffLL) return TS_ERR_UNSUPPORTED;
     const unsigned grid = (unsigned)rows;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (p->head_dim == 128)
-        ts::ts_merge_dense_kernel<128><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,
-                                                             static_cast<uint16_t *>(out), p->num_seqs, rows_all, max_splits);
-    else
-        ts::ts_merge_dense_kernel<64><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits,
-                                                            static_cast<uint16_t *>(out), p->num_seqs, rows_all, max_splits);
+    uint16_t *o = static_cast<uint16_t *>(out);
+    const bool wide = max_splits > 32;          // many parts per row: 16 warps share them
+    if (p->head_dim == 128) {
+        if (wide) ts::ts_merge_dense_kernel<128, 16><<<grid, 512, 0, s>>>(partial_o, partial_lse, num_splits, o, p->num_seqs, rows_all, max_splits);
+        else ts::ts_merge_dense_kernel<128, 4><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits, o, p->num_seqs, rows_all, max_splits);
+    } else {
+        if (wide) ts::ts_merge_dense_kernel<64, 16><<<grid, 512, 0, s>>>(partial_o, partial_lse, num_splits, o, p->num_seqs, rows_all, max_splits);
+        else ts::ts_merge_dense_kernel<64, 4><<<grid, 128, 0, s>>>(partial_o, partial_lse, num_splits, o, p->num_seqs, rows_all, max_splits);
+    }
     return cudaGetLastError() == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 
