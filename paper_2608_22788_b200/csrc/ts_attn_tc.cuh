@@ -1,22 +1,25 @@
 // Verify-attention kernel on the 5th-generation tensor cores (tcgen05 + TMEM), head_dim 128.
 //
-// Used when the (GQA group x q_len) tile of a (sequence, kv head) pair has more than 16 rows, i.e. for
-// speculative verification.  The warp-level MMA path tops out at ~550 TFLOP/s on this GPU, which
+// Used when the (GQA group x q_len) tile of a (sequence, kv head) pair has more than 16 rows (and at
+// most 128), i.e. for speculative verification.  The warp-level MMA path tops out at ~550 TFLOP/s on this GPU, which
 // is less than a 68-row tile needs to keep up with HBM; tcgen05.mma has about three times that.
 //
 // One CTA per SM = one "group" of the planner's tile line.  Roles:
-//   warp 0      TMA producer: K/V tiles (64 tokens) into a 4-stage shared-memory ring
-//   warp 1      first MMA issuer (one lane):   S[128 x 64]  = Q[128 x 128] . K^T   (8 x M128 N64 K16)
-//   warp 2      second MMA issuer (one lane):  O[128 x 128] += P[128 x 64] . V      (8 x M128 N128 K16,
+//   warp 0      TMA producer: K/V tiles (64 tokens) into a 6-stage shared-memory ring
+//   warp 1      first MMA issuer (one lane):   S[M x 64]  = Q[M x 128] . K^T   (8 x N64 K16)
+//   warp 2      second MMA issuer (one lane):  O[M x 128] += P[M x 64] . V      (8 x N128 K16,
 //               P as bf16 hi and lo).  Issuing one tcgen05.mma costs a thread 60-100 cycles here, more
 //               than these small MMAs take to execute, so the two kinds are issued by different threads.
+//               M = 64 when the pair has at most 64 rows (half of the tensor datapath then idles: the
+//               kernel is power-bound when it runs for long), else 128.
 //   warps 3..6, 7..10  two softmax warpgroups, one thread per query row (TMEM lane) each; group w
 //               takes the tiles of parity w: S is read from TMEM, masked, exponentiated; each group
 //               has its own O accumulator in TMEM, kept there for the whole segment and rescaled
 //               only when a row's running maximum grows by more than 2^8 (lazy rescale), so the
 //               common tile costs no TMEM round trip for O.  The two accumulators are merged by
-//               their (max, sum) statistics at the end of the segment.
-// There are four S/P buffers (two per softmax group): the first MMA runs two tiles ahead of the
+//               their (max, sum) statistics at the end of the segment by group 0, while group 1 fetches
+//               the next pair's Q tile.  A warp without a valid row only keeps step with the barriers.
+// There are four S/P buffers (two per softmax group): the first MMA runs up to four tiles ahead of the
 // second, so each softmax group finds its next scores ready when it finishes a tile.  P overwrites
 // S in TMEM and is the A operand of the second MMA from there.  Every mbarrier wait is bounded.
 #pragma once
