@@ -83,11 +83,15 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
                int32_t *num_splits, int32_t *status, float *part_o, float *part_lse,
                int rows_all /* q_len*Hq */, int D)
 {
-    __shared__ int warp_sums[32];
+    constexpr int kSmemB = 4096;             // up to this many sequences the prefix sums are also kept in shared
+    __shared__ int warp_sums[32];            // memory: the binary searches below are chains of dependent loads
     __shared__ int carry_s;
+    __shared__ int32_t s_cum[kSmemB + 1];
     grid_dependency_wait();      // launched ahead of the previous kernel's end: nothing is touched before this
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) { carry_s = 0; *status = TS_OK; cum_tiles[0] = 0; }
+    const bool in_smem = B <= kSmemB;
+    const int32_t *cum = in_smem ? s_cum : cum_tiles;
+    if (tid == 0) { carry_s = 0; *status = TS_OK; cum_tiles[0] = 0; s_cum[0] = 0; }
     __syncthreads();
     for (int base = 0; base < B; base += 1024) {
         const int i = base + tid;
@@ -106,21 +110,21 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
         }
         __syncthreads();
         const int incl = carry_s + x + (warp > 0 ? warp_sums[warp - 1] : 0);
-        if (i < B) cum_tiles[i + 1] = incl;
+        if (i < B) { cum_tiles[i + 1] = incl; if (in_smem) s_cum[i + 1] = incl; }
         __syncthreads();
         if (tid == 1023) carry_s = incl;
         __syncthreads();
     }
     __threadfence_block();
     __syncthreads();
-    const long long W = (long long)Hkv * cum_tiles[B];
+    const long long W = (long long)Hkv * cum[B];
 
     if (mode == kModeChunks) {
         long long want = (long long)NG * chunks_per_group;
         int chunk = (int)((W + want - 1) / want);
         if (chunk < 1) chunk = 1;
         for (int s = tid; s < B; s += 1024) {
-            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
+            const int tiles = cum[s + 1] - cum[s];
             int S = div_up(tiles, chunk);
             if (S > max_splits) S = max_splits;
             if (S < 1) S = 1;
@@ -129,7 +133,7 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
         }
         // empty sequences: their single slot is zeros / -inf
         for (int s = 0; s < B; ++s) {
-            if (cum_tiles[s + 1] != cum_tiles[s]) continue;
+            if (cum[s + 1] != cum[s]) continue;
             float *po = part_o + (size_t)s * max_splits * rows_all * D;
             float *pl = part_lse + (size_t)s * max_splits * rows_all;
             for (int i = tid; i < rows_all * D; i += 1024) po[i] = 0.f;
@@ -141,10 +145,10 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
 
     for (int k = tid; k <= NG; k += 1024) {
         long long U = (W * k) / NG;
-        int s = locate_seq(cum_tiles, B, Hkv, U);
+        int s = locate_seq(cum, B, Hkv, U);
         if (mode == kModeChunks && s < B) {
-            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
-            const long long r = U - (long long)Hkv * cum_tiles[s];
+            const int tiles = cum[s + 1] - cum[s];
+            const long long r = U - (long long)Hkv * cum[s];
             const int tau = (int)(r % tiles);
             const int ct = div_up(tiles, num_splits[s]);
             const int rem = tau % ct;
@@ -152,14 +156,14 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
                 int t2 = tau - rem + ct;
                 if (t2 > tiles) t2 = tiles;
                 U += (t2 - tau);
-                s = locate_seq(cum_tiles, B, Hkv, U);
+                s = locate_seq(cum, B, Hkv, U);
             }
         }
         GroupStart gs;
         gs.s = s; gs.g = 0; gs.tau = 0; gs.pad = 0;
         if (s < B) {
-            const int tiles = cum_tiles[s + 1] - cum_tiles[s];
-            const long long r = U - (long long)Hkv * cum_tiles[s];
+            const int tiles = cum[s + 1] - cum[s];
+            const long long r = U - (long long)Hkv * cum[s];
             gs.g = (int)(r / tiles);
             gs.tau = (int)(r % tiles);
         }
@@ -666,34 +670,48 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     const long long a0 = gpos[k_first + 1] - nx.tau, b0 = a0 + tiles;
     if (a0 < gpos[k_first]) return;                        // the pair started in an earlier group: merged there
     const int k_last = (int)((b0 * NG - 1) / W);
+    const int cnt = k_last - k_first + 1;
     for (int r = warp; r < rows; r += 4) {
         const int t = r / G, hl = r % G;
         uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
         // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
-        // (pair started before them).
-        // Groups whose piece of the tile line is empty (only when W < NG) wrote nothing: skip them.
+        // (pair started before them).  Groups whose piece of the tile line is empty (only when W < NG)
+        // wrote nothing: a piece is empty exactly when its start equals the next group's.
+        // Lane i looks at group k_first + i (+ 32, ...): the log-sum-exps come in with one round of loads.
         float M = -INFINITY;
-        for (int k = k_first; k <= k_last; ++k) {
-            if ((W * k) / NG == (W * (k + 1)) / NG) continue;
-            const size_t slot = (size_t)2 * k + (k == k_first ? 1 : 0);
-            M = fmaxf(M, part_lse[slot * rows + r]);
+        for (int b0 = 0; b0 < cnt; b0 += 32) {
+            const int k = k_first + b0 + lane;
+            float lse = -INFINITY;
+            if (k <= k_last && gpos[k] != gpos[k + 1])
+                lse = part_lse[((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r];
+            M = fmaxf(M, lse);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
         constexpr int V = D / 32;
         float acc[V];
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] = 0.f;
         float Wsum = 0.f;
         if (M != -INFINITY) {
-            for (int k = k_first; k <= k_last; ++k) {
-                if ((W * k) / NG == (W * (k + 1)) / NG) continue;
-                const size_t slot = (size_t)2 * k + (k == k_first ? 1 : 0);
-                const float lse = part_lse[slot * rows + r];
-                if (lse == -INFINITY) continue;
-                const float w = expf(lse - M);
-                Wsum += w;
-                const float *p = part_o + (slot * rows + r) * D + lane * V;
+            for (int b0 = 0; b0 < cnt; b0 += 32) {
+                const int kl = k_first + b0 + lane;
+                float wl = 0.f;
+                if (kl <= k_last && gpos[kl] != gpos[kl + 1]) {
+                    const float lse = part_lse[((size_t)2 * kl + (kl == k_first ? 1 : 0)) * rows + r];
+                    wl = lse == -INFINITY ? 0.f : expf(lse - M);
+                }
+                const int nj = cnt - b0 < 32 ? cnt - b0 : 32;
+#pragma unroll 4
+                for (int jj = 0; jj < nj; ++jj) {
+                    const float w = __shfl_sync(0xffffffffu, wl, jj);
+                    if (w == 0.f) continue;                       // empty group or empty part: not read
+                    const int k = k_first + b0 + jj;
+                    const float *p = part_o + (((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r) * D + lane * V;
+                    Wsum += w;
 #pragma unroll
-                for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+                    for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+                }
             }
         }
         const float inv = Wsum > 0.f ? 1.f / Wsum : 0.f;
