@@ -645,7 +645,7 @@ __device__ __forceinline__ void merge_row(const float *po, size_t o_stride, cons
 // by the group that holds its first part), and zero-fills the outputs of empty sequences k, k+NG, ...
 // Pairs covered by a single group were written directly by the attention kernel.
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(1024)
 ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__restrict__ gstart,
                      const long long *__restrict__ gpos, const float *__restrict__ part_o,
                      const float *__restrict__ part_lse, uint16_t *out, int B, int q_len, int Hq, int Hkv,
@@ -659,7 +659,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     for (int s0 = k_first; s0 < B; s0 += NG) {
         if (cum_tiles[s0 + 1] != cum_tiles[s0]) continue;
         uint32_t *o = reinterpret_cast<uint32_t *>(out + (size_t)s0 * q_len * Hq * D);
-        for (int i = threadIdx.x; i < q_len * Hq * D / 2; i += 128) o[i] = 0u;
+        for (int i = threadIdx.x; i < q_len * Hq * D / 2; i += blockDim.x) o[i] = 0u;
     }
     // ---- the pair cut by the end of this group's piece
     const GroupStart nx = gstart[k_first + 1];
@@ -671,7 +671,8 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     if (a0 < gpos[k_first]) return;                        // the pair started in an earlier group: merged there
     const int k_last = (int)((b0 * NG - 1) / W);
     const int cnt = k_last - k_first + 1;
-    for (int r = warp; r < rows; r += 4) {
+    const int nwarps = blockDim.x >> 5;      // one warp per output row of the pair, as many as the pair has rows
+    for (int r = warp; r < rows; r += nwarps) {
         const int t = r / G, hl = r % G;
         uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
         // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
@@ -1152,13 +1153,15 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     if (free_mode) {
         const bool overlap = env_int("TS_PDL", 1) != 0;
         const dim3 mgrid((unsigned)NG);
+        const int mwarps = a.rows < 4 ? 4 : (a.rows > 32 ? 32 : a.rows);
+        const dim3 mblock((unsigned)mwarps * 32);
         cudaError_t e;
         if (p->head_dim == 128)
-            e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles, a.gstart,
+            e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, mblock, 0, stream, overlap, a.cum_tiles, a.gstart,
                                   a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
                                   a.Hkv, NG);
         else
-            e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, dim3(128), 0, stream, overlap, a.cum_tiles, a.gstart,
+            e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, mblock, 0, stream, overlap, a.cum_tiles, a.gstart,
                                   a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
                                   a.Hkv, NG);
         if (e != cudaSuccess) return TS_ERR_CUDA;
