@@ -210,14 +210,36 @@ ts_accept_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         target_argmax[r] = (int32_t)(0xffffffffu - (uint32_t)(key & 0xffffffffull));
     }
     __syncthreads();
-    for (int b = threadIdx.x; b < B; b += blockDim.x) {
-        int a = 0;
-        while (a < gamma && draft[(long long)b * gamma + a] == target_argmax[(long long)b * R + a]) ++a;
-        accept_len[b] = a;
-        for (int i = 0; i < R; ++i) {
+    // A group of g lanes per sequence (g = the power of two that covers the gamma + 1 positions, at most
+    // 32), one lane per position: the draft and target tokens arrive with one round of loads and the first
+    // mismatch falls out of a ballot (a thread walking the block position by position paid one memory
+    // round trip per accepted token).
+    const int lane = threadIdx.x & 31;
+    int g = 1;
+    while (g < R && g < 32) g <<= 1;
+    const int per_warp = 32 / g, sub = lane / g, li = lane % g;
+    const int nslots = (blockDim.x >> 5) * per_warp;
+    const unsigned gmask = g == 32 ? 0xffffffffu : ((1u << g) - 1u);
+    for (int b0 = (threadIdx.x >> 5) * per_warp; b0 < B; b0 += nslots) {      // warp-uniform trip count
+        const int b = b0 + sub;
+        const bool live = b < B;
+        const int32_t *d = draft + (long long)(live ? b : 0) * gamma;
+        const int32_t *t = target_argmax + (long long)(live ? b : 0) * R;
+        int a = gamma;
+        bool found = false;
+        for (int i0 = 0; i0 < gamma; i0 += g) {                                // g < 32 only when gamma < g: one pass
+            const int i = i0 + li;
+            const bool miss = live && !found && i < gamma && d[i] != t[i];
+            const unsigned m = (__ballot_sync(0xffffffffu, miss) >> (sub * g)) & gmask;
+            if (m && !found) { a = i0 + __ffs(m) - 1; found = true; }
+        }
+        if (live && li == 0) accept_len[b] = a;
+        for (int i0 = 0; i0 < R; i0 += g) {
+            const int i = i0 + li;
+            if (!live || i >= R) continue;
             int32_t tok = -1;
-            if (i < a) tok = draft[(long long)b * gamma + i];
-            else if (i == a) tok = target_argmax[(long long)b * R + a];
+            if (i < a) tok = d[i];
+            else if (i == a) tok = t[i];
             out_tokens[(long long)b * R + i] = tok;
         }
     }

@@ -105,3 +105,24 @@ def test_row_stride_padding():
     torch.cuda.synchronize()
     assert rc == 0
     assert np.array_equal(tgt.cpu().numpy(), ref[0])
+
+
+@pytest.mark.parametrize("B,gamma", [(5, 1), (37, 2), (300, 3), (9, 31), (7, 32), (3, 70), (260, 0)])
+def test_block_lengths_around_the_lane_group_sizes(B, gamma):
+    # the finishing kernel gives each sequence a group of 1, 2, 4 ... 32 lanes; blocks longer than 32 positions
+    # take several passes; planted cut points anywhere in the block, including "all accepted"
+    V = 2048
+    rng = np.random.default_rng(1000 * B + gamma)
+    logits = wl.make_logits(B, gamma, V, seed=B + gamma)
+    best, _, _ = oracle.accept_greedy(logits, np.zeros((B, gamma), np.int32))
+    draft = best[:, :gamma].copy()
+    cut = rng.integers(0, gamma + 1, B)
+    for b in range(B):
+        if cut[b] < gamma:
+            draft[b, cut[b]] = (draft[b, cut[b]] + 1 + rng.integers(0, V - 1)) % V
+            later = rng.random(gamma) < 0.5                  # later positions: half still agree, half do not
+            for i in range(cut[b] + 1, gamma):
+                if later[i]:
+                    draft[b, i] = rng.integers(0, V)
+    tgt, acc, out = check(logits, draft)
+    assert np.array_equal(acc, cut)
