@@ -367,13 +367,26 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         for (int i = lane; i < R; i += 32) out[i] = -1;
         __syncwarp();
         int a = 0;
+        float ua_l = 0.f, us_l = 0.f;                  // lane l holds the uniforms and the draft of step i0 + l
+        int32_t x_l = -1;
         for (int i = 0; i <= gamma; ++i) {
+            if ((i & 31) == 0) {
+                // the next 32 steps' inputs in one round of loads (read inside the walk, each step paid a
+                // memory round trip before it could decide)
+                const int il = i + lane;
+                if (il <= gamma) {
+                    const float2 u2 = *reinterpret_cast<const float2 *>(uniforms + ((long long)b * R + il) * 2);
+                    ua_l = u2.x;
+                    us_l = u2.y;
+                    x_l = il < gamma ? draft[(long long)b * gamma + il] : -1;
+                }
+            }
             const int32_t id = s_ids[i * 32 + lane];
             const float pj = s_p[i * 32 + lane];
-            const float ua = uniforms[((long long)b * R + i) * 2], us = uniforms[((long long)b * R + i) * 2 + 1];
+            const float ua = __shfl_sync(FULL, ua_l, i & 31), us = __shfl_sync(FULL, us_l, i & 31);
             bool is_draft = false;
             if (i < gamma) {
-                const int32_t xtok = draft[(long long)b * gamma + i];
+                const int32_t xtok = __shfl_sync(FULL, x_l, i & 31);
                 is_draft = (id == xtok) && id >= 0;
                 const unsigned hit = __ballot_sync(FULL, is_draft);
                 const float px = hit ? __shfl_sync(FULL, pj, __ffs(hit) - 1) : 0.f;
