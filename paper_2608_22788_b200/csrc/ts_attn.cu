@@ -166,6 +166,15 @@ ts_plan_kernel(const int32_t *__restrict__ kv_lens, int B, int Hkv, int NG, int 
             const long long r = U - (long long)Hkv * cum[s];
             gs.g = (int)(r / tiles);
             gs.tau = (int)(r % tiles);
+            if (gs.tau != 0 && k > 0 && mode == kModeFree) {
+                // the pair under this boundary is split between group k - 1 and later ones: say so for the
+                // merge kernel -- bit 31: the pair starts inside group k - 1 (which therefore merges it),
+                // bit 30: some groups are empty (W < NG), low bits: the last group that holds a part of it
+                const long long a0 = U - gs.tau, b0 = a0 + tiles;
+                const long long prev = (W * (k - 1)) / NG;
+                const int k_last = (int)((b0 * NG - 1) / W);
+                gs.pad = (int32_t)((a0 >= prev ? 0x80000000u : 0u) | (W < NG ? 0x40000000u : 0u) | (uint32_t)k_last);
+            }
         }
         gstart[k] = gs;
         gpos[k] = U;
@@ -662,14 +671,15 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
         for (int i = threadIdx.x; i < q_len * Hq * D / 2; i += blockDim.x) o[i] = 0u;
     }
     // ---- the pair cut by the end of this group's piece
+    // (the planner left in nx.pad whether this group merges the pair, how far its parts reach, and whether
+    //  any group is empty)
     const GroupStart nx = gstart[k_first + 1];
     if (nx.s >= B || nx.tau == 0) return;                  // the piece ends on a pair boundary
+    const uint32_t info = (uint32_t)nx.pad;
+    if (!(info & 0x80000000u)) return;                     // the pair started in an earlier group: merged there
     const int s = nx.s, g = nx.g;
-    const int tiles = cum_tiles[s + 1] - cum_tiles[s];
-    const long long W = (long long)Hkv * cum_tiles[B];
-    const long long a0 = gpos[k_first + 1] - nx.tau, b0 = a0 + tiles;
-    if (a0 < gpos[k_first]) return;                        // the pair started in an earlier group: merged there
-    const int k_last = (int)((b0 * NG - 1) / W);
+    const int k_last = (int)(info & 0xffffu);
+    const bool some_empty = (info & 0x40000000u) != 0;
     const int cnt = k_last - k_first + 1;
     const int nwarps = blockDim.x >> 5;      // one warp per output row of the pair, as many as the pair has rows
     for (int r = warp; r < rows; r += nwarps) {
@@ -683,7 +693,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
         for (int b0 = 0; b0 < cnt; b0 += 32) {
             const int k = k_first + b0 + lane;
             float lse = -INFINITY;
-            if (k <= k_last && gpos[k] != gpos[k + 1])
+            if (k <= k_last && (!some_empty || gpos[k] != gpos[k + 1]))
                 lse = part_lse[((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r];
             M = fmaxf(M, lse);
         }
@@ -698,7 +708,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
             for (int b0 = 0; b0 < cnt; b0 += 32) {
                 const int kl = k_first + b0 + lane;
                 float wl = 0.f;
-                if (kl <= k_last && gpos[kl] != gpos[kl + 1]) {
+                if (kl <= k_last && (!some_empty || gpos[kl] != gpos[kl + 1])) {
                     const float lse = part_lse[((size_t)2 * kl + (kl == k_first ? 1 : 0)) * rows + r];
                     wl = lse == -INFINITY ? 0.f : expf(lse - M);
                 }
