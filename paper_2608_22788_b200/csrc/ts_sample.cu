@@ -60,20 +60,18 @@ __device__ __forceinline__ uint32_t element_key(uint32_t bits16, bool present, c
     const float y = __uint_as_float((uint32_t)rowp[idx] << 16) - pen;
     return f32_key(__float_as_uint(y));
 }
-// Register copy of a penalised logit: (logit - penalty) rounded DOWN to bf16.  Thresholds and the candidate
-// test work on these copies; rounding down keeps both sound (a bf16 threshold T is <= x iff T <= rd(x)).
-__device__ __forceinline__ uint32_t penalised_rd(uint32_t bits16, float pen)
-{
-    const float y = __uint_as_float((bits16 & 0xffffu) << 16) - pen;
-    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(y));
-}
+// Register copies of penalised logits: (logit - penalty), computed in fp32 as for the exact keys, rounded
+// to bf16.  Thresholds and the candidate test work on these copies; that is sound because the rounding is
+// monotone (if r(y) > r(x) then y > x: k copies above a threshold mean k true values above whatever lies
+// below it), and the rare candidates get their exact fp32 value back from the original logit.
 __device__ __forceinline__ void patch_vector(uint4 &x, uint32_t m, float pen)
 {
     uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        if (m & (1u << (2 * i))) w[i] = (w[i] & 0xffff0000u) | penalised_rd(w[i], pen);
-        if (m & (2u << (2 * i))) w[i] = (w[i] & 0x0000ffffu) | (penalised_rd(w[i] >> 16, pen) << 16);
+        const float lo = __uint_as_float(w[i] << 16) - ((m >> (2 * i)) & 1u ? pen : 0.f);
+        const float hi = __uint_as_float(w[i] & 0xffff0000u) - ((m >> (2 * i + 1)) & 1u ? pen : 0.f);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(hi), "f"(lo));
     }
     x = make_uint4(w[0], w[1], w[2], w[3]);
 }
