@@ -606,6 +606,16 @@ ts_attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         cc.tau += seg - 1;
         cur_advance(cc, a);
     }
+    // After a timed-out wait the loop above ran on without waiting, so copies of the last tiles may still
+    // be on their way into this CTA's shared memory: give each of them one more bounded wait before leaving.
+    if (dead) {
+        for (int t = total > ns ? total - ns : 0; t < total; ++t) {
+            const uint32_t b = bars + (t % ns) * 16;
+            const uint32_t par = (uint32_t)(t / ns) & 1u;
+            mbar_wait_bounded(b, par, a.wait_cycles);
+            mbar_wait_bounded(b + 8, par, a.wait_cycles);
+        }
+    }
 }
 
 }  // namespace ts

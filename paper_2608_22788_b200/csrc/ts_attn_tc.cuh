@@ -321,6 +321,14 @@ ts_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
             if (++st == kStages) { st = 0; if (it >= kStages) free_par ^= 1u; }
             TS_TRACE(5)
         }
+        // After a timed-out wait this warp went on issuing without waiting: give the copies of the last
+        // tiles one more bounded wait each, so that none is still writing shared memory when the CTA leaves.
+        if (dead) {
+            for (int t = total > kStages ? total - kStages : 0; t < total; ++t) {
+                mbar_wait_bounded(kfull(t % kStages), (uint32_t)(t / kStages) & 1u, a.wait_cycles);
+                mbar_wait_bounded(vfull(t % kStages), (uint32_t)(t / kStages) & 1u, a.wait_cycles);
+            }
+        }
 #ifdef TS_TC_TRACE
         if (blockIdx.x == 0 && lane == 0) {
             long long *dbg = reinterpret_cast<long long *>(a.part_o) + 128;
