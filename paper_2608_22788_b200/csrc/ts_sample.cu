@@ -253,7 +253,12 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
 #pragma unroll
         for (int i = 0; i < kThreads / 32; ++i) k8[i] = s_tkey[tid + 32 * i];
         const int want = top_k < kThreads ? top_k : kThreads;
-        uint32_t lo = 0u, hi = 65537u;                    // count(>= lo) >= want holds for lo = 0
+        // count(>= lo) >= want holds for lo = the smallest maximum (all 256 lie at or above it) and fails
+        // for hi = the largest + 1: the search runs over the spread of the maxima, not over all keys
+        uint32_t kmin = k8[0], kmax = k8[0];
+#pragma unroll
+        for (int i = 1; i < kThreads / 32; ++i) { kmin = k8[i] < kmin ? k8[i] : kmin; kmax = k8[i] > kmax ? k8[i] : kmax; }
+        uint32_t lo = __reduce_min_sync(0xffffffffu, kmin), hi = __reduce_max_sync(0xffffffffu, kmax) + 1u;
         while (hi - lo > 1u) {
             const uint32_t mid = (lo + hi) >> 1;
             int c = 0;
@@ -285,11 +290,22 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
     const int cnt = s_cnt;
     if (cnt <= kCap) {
         // ---- rank the candidates; the best top_k go out in order
-        for (int c = tid; c < cnt; c += kThreads) {
-            const unsigned long long mine = s_cand[c];
+        //      (by counting, `per` lanes to a candidate, each over a strided share of the list)
+        int per = 1;
+        while (per < 32 && cnt * per * 2 <= kThreads) per <<= 1;
+        const int sub = tid & (per - 1);
+        for (int c0 = 0; c0 < cnt; c0 += kThreads / per) {
+            const int c = c0 + tid / per;
+            const unsigned long long mine = c < cnt ? s_cand[c] : ~0ull;
             int rank = 0;
-            for (int j = 0; j < cnt; ++j) rank += s_cand[j] > mine;
-            if (rank < top_k) dst[rank] = mine;
+            int j = sub;
+            for (; j + 3 * per < cnt; j += 4 * per) {
+                const unsigned long long a0 = s_cand[j], a1 = s_cand[j + per], a2 = s_cand[j + 2 * per], a3 = s_cand[j + 3 * per];
+                rank += (int)(a0 > mine) + (int)(a1 > mine) + (int)(a2 > mine) + (int)(a3 > mine);
+            }
+            for (; j < cnt; j += per) rank += s_cand[j] > mine;
+            for (int o = per >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+            if (c < cnt && sub == 0 && rank < top_k) dst[rank] = mine;
         }
     } else {
         slow_topk(base, nvec, begin, top_k, dst, s_red, srow, &s_dh, rowp, PEN ? pen : 0.f);
