@@ -60,7 +60,8 @@ def _load():
         lib.ora_accept_sample.argtypes = [c_u16p, ctypes.c_int64, c_i32p, c_f64p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
                                           c_i32p, c_i32p, c_i32p, c_f64p, ctypes.POINTER(ctypes.c_uint8),
-                                          ctypes.c_int64, ctypes.c_double]
+                                          ctypes.c_int64, ctypes.c_double, ctypes.POINTER(ctypes.c_float),
+                                          ctypes.c_int64]
         lib.ora_rope.restype = ctypes.c_int
         lib.ora_rope.argtypes = [c_u16p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_float),
                                  ctypes.c_int64, ctypes.c_int, ctypes.c_int, c_f64p]
@@ -161,8 +162,9 @@ def accept_greedy(logits, draft, nthreads: int = 0):
 
 
 def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, top_p: float,
-                  seen=None, presence_penalty: float = 0.0):
-    """Lossless acceptance under temperature / top-k / top-p sampling with point-proposal drafts.
+                  seen=None, presence_penalty: float = 0.0, draft_probs=None):
+    """Lossless acceptance under temperature / top-k / top-p sampling; drafts are point proposals
+    unless ``draft_probs`` (float32 ``[B, gamma, V]``, the distributions they were drawn from) is given.
 
     ``logits``: uint16 bf16 bits ``[B, gamma+1, V]``; ``draft``: int ``[B, gamma]``; ``uniforms``:
     float ``[B, gamma+1, 2]`` in [0, 1).  Returns ``(accept_len [B], out_tokens [B,gamma+1],
@@ -183,6 +185,11 @@ def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, to
         sb = np.ascontiguousarray(seen, dtype=np.uint8)
         assert sb.ndim == 2 and sb.shape[0] == B and sb.shape[1] * 8 >= V
         sstride = sb.shape[1]
+    qd, qstride = None, 0
+    if draft_probs is not None:
+        qd = np.ascontiguousarray(draft_probs, dtype=np.float32)
+        assert qd.shape == (B, gamma, V)
+        qstride = V
     acc = np.empty((B,), dtype=np.int32)
     out = np.empty((B, R), dtype=np.int32)
     ids = np.empty((B, R, top_k), dtype=np.int32)
@@ -190,7 +197,8 @@ def accept_sample(logits, draft, uniforms, *, temperature: float, top_k: int, to
     rc = lib.ora_accept_sample(_p(logits, ctypes.c_uint16), V, _p(draft, ctypes.c_int32), _p(u, ctypes.c_double),
                                B, gamma, V, float(temperature), int(top_k), float(top_p),
                                _p(acc, ctypes.c_int32), _p(out, ctypes.c_int32), _p(ids, ctypes.c_int32),
-                               _p(pp, ctypes.c_double), _p(sb, ctypes.c_uint8), int(sstride), float(presence_penalty))
+                               _p(pp, ctypes.c_double), _p(sb, ctypes.c_uint8), int(sstride), float(presence_penalty),
+                               _p(qd, ctypes.c_float), int(qstride))
     if rc != 0:
         raise RuntimeError(f"ora_accept_sample failed ({rc})")
     return acc, out, ids, pp

@@ -265,13 +265,24 @@ int ora_max_threads(void)
  *                   (row i is conditioned on those drafts having been accepted).
  * The subtraction is done in single precision on the decoded logit (the precision in which a
  * serving engine holds its logits when it applies penalties).  seen == NULL: nothing seen yet.
+ *
+ * Sampled drafts (draft_probs != NULL): the drafter drew draft[b, i] from a distribution q_{b,i}
+ * over the vocabulary, given as float [B, gamma, q_row_stride >= V].  The general rule of the
+ * lossless formulation then applies at position i with p the filtered target distribution above:
+ *   - accept x iff u_accept * q(x) < p(x)              (i.e. with probability min(1, p(x) / q(x)))
+ *   - on rejection emit y drawn from norm(max(0, p - q)): weights r_j = max(0, p_j - q(id_j)) over
+ *     the kept tokens (p is zero elsewhere, so q is read at the kept tokens only), inverse CDF in
+ *     the kept order over the slots with r_j > 0; if no slot has r_j > 0 (p <= q on all of p's
+ *     support, where a rejection has probability zero) the token is drawn from p itself
+ * A one-hot q reproduces the point-proposal rule.
  */
 int ora_accept_sample(const uint16_t *logits, int64_t row_stride, const int32_t *draft,
                       const double *uniforms /* [B, gamma+1, 2] */, int B, int gamma, int V,
                       double temperature, int top_k, double top_p, int32_t *accept_len,
                       int32_t *out_tokens, int32_t *kept_ids /* [B, gamma+1, top_k] */,
                       double *kept_p /* [B, gamma+1, top_k] */, const uint8_t *seen,
-                      int64_t seen_stride, double presence_penalty)
+                      int64_t seen_stride, double presence_penalty,
+                      const float *draft_probs /* [B, gamma, q_row_stride] or NULL */, int64_t q_row_stride)
 {
     if (B < 0 || gamma < 0 || V <= 0 || top_k < 1 || !(temperature > 0.0)) return -1;
     const int R = gamma + 1;
@@ -326,6 +337,33 @@ int ora_accept_sample(const uint16_t *logits, int64_t row_stride, const int32_t 
                 const int32_t x = draft[(int64_t)b * gamma + i];
                 double px = 0.0;
                 for (int j = 0; j < top_k; ++j) if (ids[j] == x) { px = pp[j]; skip = j; }
+                if (draft_probs) {
+                    const float *q = draft_probs + ((int64_t)b * gamma + i) * q_row_stride;
+                    const double qx = (x >= 0 && x < V) ? (double)q[x] : 0.0;
+                    if (ua * qx < px) { out[i] = x; ++a; continue; }
+                    /* rejected: residual max(0, p - q) over the kept tokens */
+                    double r[top_k];
+                    double total = 0.0;
+                    for (int j = 0; j < top_k; ++j) {
+                        r[j] = 0.0;
+                        if (ids[j] < 0) continue;
+                        const double d = pp[j] - (double)q[ids[j]];
+                        if (d > 0.0) { r[j] = d; total += d; }
+                    }
+                    if (!(total > 0.0)) {            /* p <= q on the whole support: draw from p */
+                        for (int j = 0; j < top_k; ++j) if (ids[j] >= 0 && pp[j] > 0.0) { r[j] = pp[j]; total += pp[j]; }
+                    }
+                    double cum = 0.0;
+                    int32_t y = -1;
+                    for (int j = 0; j < top_k; ++j) {
+                        if (!(r[j] > 0.0)) continue;
+                        cum += r[j];
+                        y = ids[j];
+                        if (cum > us * total) break;
+                    }
+                    out[i] = y;
+                    break;
+                }
                 if (ua < px) { out[i] = x; ++a; continue; }
             }
             /* emit one token from the (residual) distribution and stop */

@@ -224,3 +224,168 @@ def test_large_presence_penalty_removes_seen_tokens_from_the_kept_set():
         kept = set(ids[b][ids[b] >= 0].tolist())
         assert not (kept & set(seen_tokens[b]))
         assert acc[b] == 0                                      # the drafts are seen tokens: never kept, rejected
+
+
+# ------------------------------------------------------------------ sampled drafts (general proposal q)
+def brute_accept_q(logits_bits, draft, u, q, temperature, top_k, top_p):
+    """The general rule written independently: accept with probability min(1, p/q), else draw from
+    norm(max(0, p - q)) over the whole vocabulary (dense vectors, no kept-slot bookkeeping)."""
+    f = wl.bf16_bits_to_f32(logits_bits).astype(np.float64)
+    B, R, V = f.shape
+    gamma = R - 1
+    acc = np.zeros(B, np.int32)
+    out = np.full((B, R), -1, np.int32)
+    for b in range(B):
+        for i in range(R):
+            ids, pk = filtered_distribution(f[b, i], temperature, top_k, top_p)
+            p = np.zeros(V)
+            p[ids] = pk
+            if i < gamma:
+                x = int(draft[b, i])
+                qv = q[b, i].astype(np.float64)
+                if u[b, i, 0] * qv[x] < p[x]:
+                    out[b, i] = x
+                    acc[b] += 1
+                    continue
+                w = np.maximum(p - qv, 0.0)
+                if not w.sum() > 0:
+                    w = p
+            else:
+                w = p
+            order = [t for t in ids if w[t] > 0]            # inverse CDF runs in the kept order
+            total = sum(w[t] for t in order)
+            cum, y = 0.0, -1
+            for t in order:
+                cum += w[t]
+                y = t
+                if cum > u[b, i, 1] * total:
+                    break
+            out[b, i] = y
+            break
+    return acc, out
+
+
+def _random_q(rng, B, gamma, V, logits, sharp):
+    """Proposal distributions loosely correlated with the target: softmax of the logits plus noise."""
+    f = wl.bf16_bits_to_f32(logits)[:, :gamma].astype(np.float64)
+    z = sharp * f + rng.standard_normal((B, gamma, V))
+    z -= z.max(-1, keepdims=True)
+    q = np.exp(z)
+    q /= q.sum(-1, keepdims=True)
+    return q.astype(np.float32)
+
+
+def _draw(rng, q):
+    B, gamma, V = q.shape
+    d = np.zeros((B, gamma), np.int32)
+    for b in range(B):
+        for i in range(gamma):
+            pr = q[b, i].astype(np.float64)
+            d[b, i] = rng.choice(V, p=pr / pr.sum())
+    return d
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_sampled_drafts_match_numpy_bruteforce(seed):
+    rng = np.random.default_rng(100 + seed)
+    B, gamma, V = 6, 4, 160
+    logits = wl.make_logits(B, gamma, V, seed=seed)
+    q = _random_q(rng, B, gamma, V, logits, sharp=[1.4, 0.5, 2.5, 1.0, 1.4, 0.0][seed])
+    draft = _draw(rng, q)
+    u = rng.random((B, gamma + 1, 2))
+    T, k, pnuc = [(0.7, 20, 0.8), (1.0, 5, 0.95), (0.3, 20, 1.0), (2.0, 50, 0.5), (0.7, 1, 0.8), (0.7, 20, 0.8)][seed]
+    acc, out, _, _ = oracle.accept_sample(logits, draft, u, temperature=T, top_k=k, top_p=pnuc, draft_probs=q)
+    racc, rout = brute_accept_q(logits, draft, u, q, T, k, pnuc)
+    assert np.array_equal(acc, racc) and np.array_equal(out, rout)
+    assert acc.max() > 0 or seed == 5
+
+
+def test_one_hot_proposal_is_the_point_proposal_rule():
+    rng = np.random.default_rng(7)
+    B, gamma, V = 12, 5, 700
+    logits = wl.make_logits(B, gamma, V, seed=3)
+    best = np.argmax(wl.bf16_bits_to_f32(logits), -1)
+    draft = np.where(rng.random((B, gamma)) < 0.7, best[:, :gamma], rng.integers(0, V, (B, gamma))).astype(np.int32)
+    q = np.zeros((B, gamma, V), np.float32)
+    np.put_along_axis(q, draft[..., None].astype(np.int64), 1.0, axis=-1)
+    u = rng.random((B, gamma + 1, 2))
+    kw = dict(temperature=0.7, top_k=20, top_p=0.8)
+    a0, o0, _, _ = oracle.accept_sample(logits, draft, u, **kw)
+    a1, o1, _, _ = oracle.accept_sample(logits, draft, u, draft_probs=q, **kw)
+    assert np.array_equal(a0, a1) and np.array_equal(o0, o1)
+    assert a0.min() < gamma and a0.max() > 0
+
+
+def test_sampled_draft_closed_form():
+    # p = (1/2, 1/4, 1/4) as above; q = (1/4, 1/2, 1/4)
+    T = 1.0 / math.log(2.0)
+    logits = _bits(np.array([[[1.0, 0.0, 0.0], [1.0, 0.0, 0.0]]]))
+    q = np.array([[[0.25, 0.5, 0.25]]], np.float32)
+
+    def run(draft, ua, us):
+        u = np.array([[[ua, us], [0.0, us]]])
+        acc, out, _, _ = oracle.accept_sample(logits, [[draft]], u, temperature=T, top_k=3, top_p=1.0, draft_probs=q)
+        return int(acc[0]), out[0].tolist()
+
+    assert run(0, 0.999, 0.1) == (1, [0, 0])        # p/q = 2: always accepted; bonus token 0 at 0.1
+    assert run(2, 0.999, 0.6) == (1, [2, 1])        # p/q = 1: accepted for every u < 1
+    assert run(1, 0.499, 0.8) == (1, [1, 2])        # p/q = 1/2: accepted below 1/2 ...
+    assert run(1, 0.501, 0.0) == (0, [0, -1])       # ... rejected above; max(0, p - q) = (1/4, 0, 0): token 0
+    assert run(1, 0.501, 0.999) == (0, [0, -1])
+
+
+def test_proposal_equal_to_target_is_always_accepted():
+    rng = np.random.default_rng(9)
+    B, gamma, V = 8, 6, 300
+    logits = wl.make_logits(B, gamma, V, seed=9)
+    f = wl.bf16_bits_to_f32(logits).astype(np.float64)
+    q = np.zeros((B, gamma, V), np.float32)
+    # temperature 1 and powers of two would make p exact in float32; in general q = float32(p) differs
+    # from p by rounding, so u is kept away from 1
+    for b in range(B):
+        for i in range(gamma):
+            ids, p = filtered_distribution(f[b, i], 0.7, 20, 0.8)
+            q[b, i, ids] = p
+    draft = _draw(rng, q)
+    u = rng.random((B, gamma + 1, 2)) * 0.999
+    acc, out, _, _ = oracle.accept_sample(logits, draft, u, temperature=0.7, top_k=20, top_p=0.8, draft_probs=q)
+    assert (acc == gamma).all() and np.array_equal(out[:, :gamma], draft)
+
+
+def test_sampled_drafts_are_lossless():
+    # sum over draft tokens x of q(x) * P(emit y | draft x) = p(y): the lattice over (u_accept, u_sample)
+    # integrates the inner probability, the sum over x is exact
+    rng = np.random.default_rng(4)
+    V, N = 6, 300
+    x = rng.standard_normal((1, 2, V)).astype(np.float32) * 2
+    logits = _bits(x)
+    T, k, pnuc = 0.9, 4, 0.95
+    ids, p = filtered_distribution(wl.bf16_bits_to_f32(logits)[0, 0].astype(np.float64), T, k, pnuc)
+    want = np.zeros(V)
+    want[ids] = p
+    qv = rng.dirichlet(np.ones(V)).astype(np.float32)
+    grid = (np.arange(N) + 0.5) / N
+    ua, us = np.meshgrid(grid, grid, indexing="ij")
+    u = np.zeros((N * N, 2, 2))
+    u[:, 0, 0], u[:, 0, 1] = ua.ravel(), us.ravel()
+    big = np.broadcast_to(logits, (N * N, 2, V)).copy()
+    qq = np.broadcast_to(qv, (N * N, 1, V)).copy()
+    mix = np.zeros(V)
+    rejected_somewhere = False
+    for tok in range(V):
+        acc, out, _, _ = oracle.accept_sample(big, np.full((N * N, 1), tok), u, temperature=T, top_k=k, top_p=pnuc,
+                                              draft_probs=qq)
+        rejected_somewhere |= bool((acc == 0).any())
+        mix += float(qv[tok]) * np.bincount(out[:, 0], minlength=V) / (N * N)
+    assert rejected_somewhere
+    assert np.abs(mix - want).max() <= 2.5 / N
+
+
+def test_unnormalised_proposal_above_target_falls_back_to_the_target():
+    # q = 2 p is not a distribution; a rejection then leaves no positive residual and the token comes from p
+    T = 1.0 / math.log(2.0)
+    logits = _bits(np.array([[[1.0, 0.0, 0.0], [1.0, 0.0, 0.0]]]))
+    q = np.array([[[1.0, 0.5, 0.5]]], np.float32)
+    u = np.array([[[0.9, 0.6], [0.0, 0.0]]])
+    acc, out, _, _ = oracle.accept_sample(logits, [[0]], u, temperature=T, top_k=3, top_p=1.0, draft_probs=q)
+    assert int(acc[0]) == 0 and out[0].tolist() == [1, -1]      # cumulative (1/2, 3/4, 1): 0.6 picks token 1
