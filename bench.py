@@ -203,11 +203,18 @@ class Sample:
     """ts_accept_sample on the same logits / drafts as an Accept instance (paper's sampling regime)."""
 
     def __init__(self, acc: "Accept", seed=0, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=0.0,
-                 seen_density=0.0):
+                 seen_density=0.0, proposal=False):
         import torch
         self.api, self.acc = acc.api, acc
         self.kw = dict(temperature=temperature, top_k=top_k, top_p=top_p)
         rng = np.random.default_rng([seed, 17])
+        if proposal and acc.gamma > 0:
+            # sampled drafts: a proposal distribution per draft position, here the softmax of the target's own
+            # logits at a slightly higher temperature, made on the device.  The drafts themselves stay as they
+            # are: the kernel reads q at the draft token and at the kept tokens only, whatever drew the draft
+            lg = acc.logits[:, :acc.gamma].float()
+            self.kw.update(draft_probs=torch.softmax(lg / (temperature * 1.2), dim=-1).contiguous())
+            del lg
         if presence_penalty != 0.0:
             # seen-token bitmap: each sequence has generated `seen_density` of the vocabulary so far
             bits = np.random.default_rng([seed, 18]).random((acc.B, acc.V)) < seen_density
@@ -615,7 +622,13 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         record(f"verify_g{g}:ts_accept_sample_penalized", acc.bytes, pmed, pmn, int((pen.alen + 1).sum().item()),
                {"temperature": 0.7, "top_k": 20, "top_p": 0.8, "presence_penalty": 1.5,
                 "note": "seen-token bitmap with 3 % of the vocabulary set (about 4500 distinct generated tokens)"})
-        del acc, smp, pen
+        prop = Sample(acc, seed=seed, presence_penalty=1.5, seen_density=0.03, proposal=True)
+        qmed, qmn = time_with_flush(prop.run, flush)
+        record(f"verify_g{g}:ts_accept_sample_proposal", acc.bytes, qmed, qmn, int((prop.alen + 1).sum().item()),
+               {"temperature": 0.7, "top_k": 20, "top_p": 0.8, "presence_penalty": 1.5,
+                "note": "sampled-draft rule with a proposal distribution fp32 [16, gamma, vocab]; it is read at the "
+                        "draft token and the kept tokens only, so the credited bytes are the logits'"})
+        del acc, smp, pen, prop
 
     # route-specific draft depths (Section 4.3: a shallow depth on the wide bulk pool, a deep one on the
     # narrow tail pool, the two summing to twice the base depth): verify attention on the bulk batch

@@ -242,6 +242,30 @@ int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int
                                int32_t *out_tokens, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * ts_accept_sample_penalized for drafters that SAMPLE their tokens: draft[b, i] was drawn from a
+ * proposal distribution q_{b,i} over the vocabulary, and the general rule of the lossless formulation
+ * the paper adopts (Section 3.4) applies, with p the filtered target distribution of row (b, i):
+ *   x_i is accepted iff u_accept * q(x_i) < p(x_i), i.e. with probability min(1, p(x_i) / q(x_i));
+ *   at the first rejection one token is drawn from norm(max(0, p - q)) -- weights max(0, p_j - q(j))
+ *   over the kept tokens j in their order, since p is zero elsewhere -- and the walk stops.  If that
+ *   leaves no positive weight (p <= q on all of p's support: a rejection then has probability zero
+ *   for a normalised q, but a caller may pass an unnormalised one) the token is drawn from p itself.
+ *   draft_probs             fp32, q_{b,i} at draft_probs + (b*gamma+i)*draft_probs_row_stride, vocab
+ *                           entries each; read at the draft token and at the at most top_k kept
+ *                           tokens of the row only (no extra pass over the vocabulary); device memory
+ *   draft_probs_row_stride  in elements, >= vocab
+ * draft_probs == NULL is the point-proposal rule (q = one-hot at the draft token), i.e.
+ * ts_accept_sample_penalized exactly; a one-hot draft_probs gives the same decisions.  A draft token
+ * outside [0, vocab) is rejected.  Everything else as ts_accept_sample_penalized.
+ */
+int ts_accept_sample_proposal(const void *logits, int64_t row_stride, const int32_t *draft,
+                              const float *draft_probs, int64_t draft_probs_row_stride, const float *uniforms,
+                              int32_t num_seqs, int32_t gamma, int32_t vocab, float temperature, int32_t top_k,
+                              float top_p, float presence_penalty, const uint8_t *seen, int64_t seen_stride,
+                              int32_t *accept_len, int32_t *out_tokens, void *workspace, size_t workspace_bytes,
+                              void *stream);
+
+/*
  * ts_accept_greedy for callers that have no device memory to give and cannot get any.  (The paper
  * has no counterpart; this is a packaging variant of ts_accept_greedy.)  Who that is: a serving
  * process that handed all of HBM to its KV cache at start-up and kept no allocator for side

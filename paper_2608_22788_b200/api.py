@@ -22,7 +22,7 @@ TS_OK = 0
 EXPORTED_SYMBOLS = (
     "ts_attn_workspace_bytes", "ts_splitkv_workspace_bytes", "ts_decode_attn", "ts_verify_attn",
     "ts_decode_attn_splitkv", "ts_lse_merge", "ts_accept_workspace_bytes", "ts_accept_greedy",
-    "ts_accept_greedy_noalloc", "ts_sample_workspace_bytes", "ts_accept_sample", "ts_accept_sample_penalized", "ts_kv_append", "ts_rope_kv_append",
+    "ts_accept_greedy_noalloc", "ts_sample_workspace_bytes", "ts_accept_sample", "ts_accept_sample_penalized", "ts_accept_sample_proposal", "ts_kv_append", "ts_rope_kv_append",
     "ts_set_attn_timing_events", "ts_status_string",
 )
 
@@ -80,6 +80,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ts_accept_sample_penalized.restype = ctypes.c_int
     lib.ts_accept_sample_penalized.argtypes = [vp, i64, vp, vp, i32, i32, i32, ctypes.c_float, i32, ctypes.c_float,
                                                ctypes.c_float, vp, i64, vp, vp, vp, sz, vp]
+    lib.ts_accept_sample_proposal.restype = ctypes.c_int
+    lib.ts_accept_sample_proposal.argtypes = [vp, i64, vp, vp, i64, vp, i32, i32, i32, ctypes.c_float, i32, ctypes.c_float,
+                                              ctypes.c_float, vp, i64, vp, vp, vp, sz, vp]
     lib.ts_kv_append.restype = ctypes.c_int
     lib.ts_kv_append.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
     lib.ts_rope_kv_append.restype = ctypes.c_int
@@ -247,16 +250,39 @@ def sample_workspace_bytes(num_seqs: int, gamma: int, vocab: int, top_k: int) ->
 
 
 def ts_accept_sample(logits, draft, uniforms, accept_len, out_tokens, workspace, *, temperature: float, top_k: int,
-                     top_p: float, row_stride=None, presence_penalty: float = 0.0, seen=None):
+                     top_p: float, row_stride=None, presence_penalty: float = 0.0, seen=None, draft_probs=None):
     """Lossless draft acceptance under temperature / top-k / top-p sampling (see the header).
 
     With ``presence_penalty`` (and optionally ``seen``, a uint8 bitmap ``[B, >= V/8]`` of the tokens
-    each sequence has generated so far) the call goes through ``ts_accept_sample_penalized``.
+    each sequence has generated so far) the call goes through ``ts_accept_sample_penalized``; with
+    ``draft_probs`` (float32 ``[B, gamma, >= V]``, the distributions the drafts were sampled from)
+    through ``ts_accept_sample_proposal``.
     """
     lib = load_library()
     B, R, V = logits.shape
     gamma = R - 1
     stride = int(row_stride) if row_stride is not None else int(logits.stride(1))
+    if draft_probs is not None:
+        if draft_probs.dtype != torch.float32 or draft_probs.dim() != 3 or draft_probs.shape[0] != B \
+                or draft_probs.shape[1] != gamma or draft_probs.stride(2) != 1:
+            raise TailSieveError("draft_probs must be float32 [num_seqs, gamma, vocab] with unit inner stride")
+        if gamma > 1 and draft_probs.stride(0) != gamma * draft_probs.stride(1):
+            raise TailSieveError("draft_probs rows must be evenly strided")
+        seen_stride = 0
+        if seen is not None:
+            if seen.dtype != torch.uint8 or seen.dim() != 2 or seen.shape[0] != B:
+                raise TailSieveError("seen must be a uint8 bitmap [num_seqs, bytes]")
+            seen_stride = int(seen.stride(0))
+        q_stride = int(draft_probs.stride(1)) if gamma > 0 else V
+        rc = lib.ts_accept_sample_proposal(_ptr(logits, "logits"), stride, _ptr(draft, "draft") if gamma > 0 else None,
+                                           _ptr(draft_probs, "draft_probs") if gamma > 0 else None, q_stride,
+                                           _ptr(uniforms, "uniforms"), B, gamma, V, float(temperature), int(top_k),
+                                           float(top_p), float(presence_penalty), _ptr(seen, "seen"), seen_stride,
+                                           _ptr(accept_len, "accept_len"), _ptr(out_tokens, "out_tokens"),
+                                           _ptr(workspace, "workspace"), workspace.numel() * workspace.element_size(),
+                                           _stream())
+        _check(rc, "ts_accept_sample_proposal")
+        return accept_len, out_tokens
     if presence_penalty == 0.0 and seen is None:
         rc = lib.ts_accept_sample(_ptr(logits, "logits"), stride, _ptr(draft, "draft") if gamma > 0 else None,
                                   _ptr(uniforms, "uniforms"), B, gamma, V, float(temperature), int(top_k), float(top_p),

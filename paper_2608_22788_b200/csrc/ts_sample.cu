@@ -318,6 +318,7 @@ __global__ void __launch_bounds__(1024)
 ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks, int top_k,
                         const int32_t *__restrict__ draft,
                         const float *__restrict__ uniforms, int gamma, float inv_temperature, float top_p,
+                        const float *__restrict__ draft_probs, long long q_stride, int vocab,
                         int32_t *accept_len, int32_t *out_tokens)
 {
     extern __shared__ unsigned char smem[];
@@ -327,7 +328,8 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
     const int total = chunks * top_k;
     int32_t *s_ids = reinterpret_cast<int32_t *>(smem);                       // [R][32]
     float *s_p = reinterpret_cast<float *>(smem + (size_t)R * 32 * 4);         // [R][32]
-    unsigned long long *s_best = reinterpret_cast<unsigned long long *>(smem + (size_t)R * 32 * 8);   // [warps][32]
+    float *s_q = reinterpret_cast<float *>(smem + (size_t)R * 32 * 8);         // [R][32]: proposal at the kept tokens
+    unsigned long long *s_best = reinterpret_cast<unsigned long long *>(smem + (size_t)R * 32 * 12);  // [warps][32]
     unsigned long long *s_cand = s_best + nwarps * 32;                         // [warps][chunks * top_k]
     grid_dependency_wait();       // the chunk keys of the kernel before
     const int b = blockIdx.x;
@@ -374,6 +376,9 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         for (int o = 16; o > 0; o >>= 1) ks += __shfl_xor_sync(FULL, ks, o);
         s_ids[i * 32 + lane] = kept ? idx : -1;
         s_p[i * 32 + lane] = kept ? p / ks : 0.f;
+        // sampled drafts: the proposal is needed at the kept tokens only (the target is zero elsewhere)
+        if (draft_probs && i < gamma)
+            s_q[i * 32 + lane] = kept ? draft_probs[((long long)b * gamma + i) * q_stride + idx] : 0.f;
     }
     __syncthreads();
     if (warp == 0) {
@@ -383,6 +388,7 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         int a = 0;
         float ua_l = 0.f, us_l = 0.f;                  // lane l holds the uniforms and the draft of step i0 + l
         int32_t x_l = -1;
+        float qx_l = 1.f;                              // proposal probability of that draft (1: point proposal)
         for (int i = 0; i <= gamma; ++i) {
             if ((i & 31) == 0) {
                 // the next 32 steps' inputs in one round of loads (read inside the walk, each step paid a
@@ -393,6 +399,8 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
                     ua_l = u2.x;
                     us_l = u2.y;
                     x_l = il < gamma ? draft[(long long)b * gamma + il] : -1;
+                    if (draft_probs && il < gamma)
+                        qx_l = (x_l >= 0 && x_l < vocab) ? draft_probs[((long long)b * gamma + il) * q_stride + x_l] : 0.f;
                 }
             }
             const int32_t id = s_ids[i * 32 + lane];
@@ -404,10 +412,29 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
                 is_draft = (id == xtok) && id >= 0;
                 const unsigned hit = __ballot_sync(FULL, is_draft);
                 const float px = hit ? __shfl_sync(FULL, pj, __ffs(hit) - 1) : 0.f;
-                if (ua < px) {                      // accepted: next position
+                const float qx = __shfl_sync(FULL, qx_l, i & 31);
+                if (ua * qx < px) {                 // accepted (probability min(1, p / q)): next position
                     if (lane == 0) out[i] = xtok;
                     ++a;
                     continue;
+                }
+                if (draft_probs) {
+                    // rejected: one token from norm(max(0, p - q)); from p itself if nothing is left of it
+                    float r = id >= 0 ? fmaxf(pj - s_q[i * 32 + lane], 0.f) : 0.f;
+                    if (!__ballot_sync(FULL, r > 0.f)) r = id >= 0 ? pj : 0.f;
+                    float cum = r, tot = r;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const float y = __shfl_up_sync(FULL, cum, o); if (lane >= o) cum += y; }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(FULL, tot, o);
+                    const unsigned over = __ballot_sync(FULL, r > 0.f && cum > us * tot);
+                    const unsigned lives = __ballot_sync(FULL, r > 0.f);
+                    int pick = -1;
+                    if (over) pick = __ffs(over) - 1;
+                    else if (lives) pick = 31 - __clz(lives);
+                    const int32_t y = pick >= 0 ? __shfl_sync(FULL, id, pick) : -1;
+                    if (lane == 0) out[i] = y;
+                    break;
                 }
             }
             // one token from the (residual) distribution, then stop
@@ -471,7 +498,19 @@ int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int
                                int32_t *accept_len, int32_t *out_tokens, void *workspace, size_t workspace_bytes,
                                void *stream)
 {
+    return ts_accept_sample_proposal(logits, row_stride, draft, nullptr, 0, uniforms, num_seqs, gamma, vocab, temperature,
+                                     top_k, top_p, presence_penalty, seen, seen_stride, accept_len, out_tokens, workspace,
+                                     workspace_bytes, stream);
+}
+
+int ts_accept_sample_proposal(const void *logits, int64_t row_stride, const int32_t *draft, const float *draft_probs,
+                              int64_t draft_probs_row_stride, const float *uniforms, int32_t num_seqs, int32_t gamma,
+                              int32_t vocab, float temperature, int32_t top_k, float top_p, float presence_penalty,
+                              const uint8_t *seen, int64_t seen_stride, int32_t *accept_len, int32_t *out_tokens,
+                              void *workspace, size_t workspace_bytes, void *stream)
+{
     using namespace ts::smp;
+    if (draft_probs && draft_probs_row_stride < vocab) return TS_ERR_INVALID_ARG;
     if (isnan(presence_penalty) || isinf(presence_penalty)) return TS_ERR_INVALID_ARG;
     if (seen && seen_stride * 8 < vocab) return TS_ERR_INVALID_ARG;
     if (num_seqs < 0 || gamma < 0 || vocab < 1) return TS_ERR_INVALID_ARG;
@@ -509,7 +548,7 @@ int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int
     int warps = R < 32 ? R : 32;
     size_t smem;
     for (;;) {
-        smem = (size_t)R * 32 * 8 + (size_t)warps * 32 * 8 + (size_t)warps * chunks * top_k * 8;
+        smem = (size_t)R * 32 * 12 + (size_t)warps * 32 * 8 + (size_t)warps * chunks * top_k * 8;
         if (smem <= 48 * 1024 || warps == 1) break;
         warps = (warps + 1) / 2;
     }
@@ -518,7 +557,8 @@ int ts_accept_sample_penalized(const void *logits, int64_t row_stride, const int
     const bool overlap = !(pdl && pdl[0] == '0');
     const cudaError_t e = ts::launch_overlapped(ts_sample_finish_kernel, dim3((unsigned)num_seqs), dim3(warps * 32), smem, s,
                                                 overlap, (const unsigned long long *)keys, chunks, (int)top_k, draft,
-                                                uniforms, (int)gamma, 1.0f / temperature, top_p, accept_len, out_tokens);
+                                                uniforms, (int)gamma, 1.0f / temperature, top_p, draft_probs,
+                                                (long long)draft_probs_row_stride, (int)vocab, accept_len, out_tokens);
     return e == cudaSuccess ? TS_OK : TS_ERR_CUDA;
 }
 

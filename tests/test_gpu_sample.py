@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 MARGIN = 1e-5
 
 
-def run_gpu(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0):
+def run_gpu(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0, q=None):
     B, R, V = logits_bits.shape
     gamma = R - 1
     lg = torch.from_numpy(np.ascontiguousarray(logits_bits).view(np.int16)).cuda().view(torch.bfloat16)
@@ -27,16 +27,33 @@ def run_gpu(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0):
     out = torch.full((B, R), -5, dtype=torch.int32, device="cuda")
     ws = torch.empty(api.sample_workspace_bytes(B, gamma, V, k), dtype=torch.uint8, device="cuda")
     sd = torch.from_numpy(np.ascontiguousarray(seen)).cuda() if seen is not None else None
-    api.ts_accept_sample(lg, dr, uu, acc, out, ws, temperature=T, top_k=k, top_p=pnuc, presence_penalty=pen, seen=sd)
+    qd = torch.from_numpy(np.ascontiguousarray(q, dtype=np.float32)).cuda() if q is not None else None
+    api.ts_accept_sample(lg, dr, uu, acc, out, ws, temperature=T, top_k=k, top_p=pnuc, presence_penalty=pen, seen=sd,
+                         draft_probs=qd)
     torch.cuda.synchronize()
     return acc.cpu().numpy(), out.cpu().numpy()
 
 
-def near_tie(b, i, draft, u, ids, pp, gamma, pnuc):
+def near_tie(b, i, draft, u, ids, pp, gamma, pnuc, q=None):
     """True if some comparison at row (b, i) is within MARGIN in the oracle's arithmetic."""
     p = pp[b, i]
     kept = ids[b, i] >= 0
     ua, us = u[b, i]
+    if q is not None and i < gamma:
+        # sampled draft: u_accept * q(x) against p(x), then the inverse CDF over max(0, p - q); the fp32
+        # differences p - q carry an absolute error of a few 1e-7, whatever their size
+        x = int(draft[b, i])
+        qv = q[b, i].astype(np.float64)
+        px = p[ids[b, i] == x].sum()
+        if abs(ua * qv[x] - px) < MARGIN:
+            return True
+        r = np.where(kept, np.maximum(p - qv[np.maximum(ids[b, i], 0)], 0.0), 0.0)
+        if (np.abs(np.where(kept, p - qv[np.maximum(ids[b, i], 0)], 1.0)) < 1e-6).any():
+            return True                                  # a slot on the edge of the residual's support
+        tot = r.sum()
+        if tot > 0 and (np.abs(np.cumsum(r) - us * tot) < 4e-6).any():
+            return True
+        return False
     # nucleus boundary (needs the unrenormalised cumulative sums: recompute is overkill; use a proxy:
     # the kept mass before renormalisation cannot be told from here, so only flag exact-looking cases)
     if i < gamma:
@@ -54,19 +71,19 @@ def near_tie(b, i, draft, u, ids, pp, gamma, pnuc):
     return False
 
 
-def check(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0):
+def check(logits_bits, draft, u32, T, k, pnuc, seen=None, pen=0.0, q=None):
     B, R, V = logits_bits.shape
     gamma = R - 1
     u = np.asarray(u32, np.float32)
     racc, rout, ids, pp = oracle.accept_sample(logits_bits, draft, u.astype(np.float64), temperature=T, top_k=k, top_p=pnuc,
-                                               seen=seen, presence_penalty=pen)
-    gacc, gout = run_gpu(logits_bits, draft, u, T, k, pnuc, seen, pen)
+                                               seen=seen, presence_penalty=pen, draft_probs=q)
+    gacc, gout = run_gpu(logits_bits, draft, u, T, k, pnuc, seen, pen, q)
     undecided = 0
     for b in range(B):
         if gacc[b] == racc[b] and np.array_equal(gout[b], rout[b]):
             continue
         last = min(int(racc[b]), int(gacc[b]))
-        if any(near_tie(b, i, np.asarray(draft).reshape(B, gamma), u, ids, pp, gamma, pnuc) for i in range(last + 1)):
+        if any(near_tie(b, i, np.asarray(draft).reshape(B, gamma), u, ids, pp, gamma, pnuc, q) for i in range(last + 1)):
             undecided += 1
             continue
         raise AssertionError(f"sequence {b}: gpu accept {gacc[b]} tokens {gout[b]} vs oracle {racc[b]} {rout[b]}")
@@ -218,3 +235,86 @@ def test_presence_penalty_argument_errors():
         api.ts_accept_sample(lg, None, u, acc, out, ws, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=1.5, seen=short)
     with pytest.raises(api.TailSieveError):
         api.ts_accept_sample(lg, None, u, acc, out, ws, temperature=0.7, top_k=20, top_p=0.8, presence_penalty=float("nan"))
+
+
+# ------------------------------------------------------------------ sampled drafts (proposal distribution q)
+def _proposal(rng, logits, gamma, sharp):
+    """q = softmax(sharp * logits + noise) per draft position, float32, and one draw from each."""
+    f = wl.bf16_bits_to_f32(logits)[:, :gamma].astype(np.float32)
+    z = sharp * f + rng.standard_normal(f.shape, dtype=np.float32)
+    z -= z.max(-1, keepdims=True)
+    q = np.exp(z)
+    q /= q.sum(-1, keepdims=True)
+    B, _, V = q.shape
+    c = np.cumsum(q.astype(np.float64), -1)
+    draws = rng.random((B, gamma, 1)) * c[..., -1:]
+    draft = np.minimum((c < draws).sum(-1), V - 1).astype(np.int32)
+    return q.astype(np.float32), draft
+
+
+@pytest.mark.parametrize("gamma", [4, 16])
+def test_sampled_drafts_full_vocab(gamma):
+    B, V = 16, wl.VOCAB
+    rng = np.random.default_rng(50 + gamma)
+    logits = wl.make_logits(B, gamma, V, seed=60 + gamma)
+    q, draft = _proposal(rng, logits, gamma, sharp=1.0 / 0.7)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    acc, out = check(logits, draft, u, 0.7, 20, 0.8, q=q)
+    assert acc.max() > 0 and acc.min() < gamma
+
+
+@pytest.mark.parametrize("cfg", [(1.0, 5, 0.95, 1.0), (0.3, 32, 1.0, 2.0), (2.0, 32, 0.5, 0.3), (0.7, 1, 0.8, 1.4), (0.7, 20, 0.8, 0.0)])
+def test_sampled_drafts_other_parameters(cfg):
+    T, k, pnuc, sharp = cfg
+    B, gamma, V = 48, 3, 4096
+    rng = np.random.default_rng(int(T * 10) + k + 7)
+    logits = wl.make_logits(B, gamma, V, seed=k + 1)
+    q, draft = _proposal(rng, logits, gamma, sharp)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    check(logits, draft, u, T, k, pnuc, q=q)
+
+
+def test_one_hot_proposal_gives_the_point_proposal_results():
+    B, gamma, V = 16, 8, 32768
+    rng = np.random.default_rng(8)
+    logits = wl.make_logits(B, gamma, V, seed=8)
+    best = np.argmax(wl.bf16_bits_to_f32(logits), -1)
+    draft = np.where(rng.random((B, gamma)) < 0.8, best[:, :gamma], rng.integers(0, V, (B, gamma))).astype(np.int32)
+    q = np.zeros((B, gamma, V), np.float32)
+    np.put_along_axis(q, draft[..., None].astype(np.int64), 1.0, axis=-1)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    a0, o0 = run_gpu(logits, draft, u, 0.7, 20, 0.8)
+    a1, o1 = run_gpu(logits, draft, u, 0.7, 20, 0.8, q=q)
+    assert np.array_equal(a0, a1) and np.array_equal(o0, o1)
+
+
+def test_sampled_drafts_with_the_presence_penalty():
+    B, gamma, V = 24, 5, 8192
+    rng = np.random.default_rng(12)
+    logits = wl.make_logits(B, gamma, V, seed=12)
+    q, draft = _proposal(rng, logits, gamma, sharp=1.4)
+    seen = rng.integers(0, 256, (B, V // 8), dtype=np.uint8) & rng.integers(0, 256, (B, V // 8), dtype=np.uint8)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    check(logits, draft, u, 0.7, 20, 0.8, seen=seen, pen=1.5, q=q)
+
+
+def test_proposal_equal_to_target_accepts_everything_and_out_of_range_draft_is_rejected():
+    B, gamma, V = 8, 4, 2048
+    rng = np.random.default_rng(3)
+    logits = wl.make_logits(B, gamma, V, seed=3)
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32) * 0.99
+    _, _, ids, pp = oracle.accept_sample(logits, np.zeros((B, gamma), np.int32), u.astype(np.float64), temperature=0.7,
+                                         top_k=20, top_p=0.8)
+    q = np.zeros((B, gamma, V), np.float32)
+    draft = np.zeros((B, gamma), np.int32)
+    for b in range(B):
+        for i in range(gamma):
+            kept = ids[b, i] >= 0
+            q[b, i, ids[b, i][kept]] = pp[b, i][kept]
+            draft[b, i] = ids[b, i][rng.integers(0, kept.sum())]
+    acc, out = run_gpu(logits, draft, u, 0.7, 20, 0.8, q=q)
+    assert (acc == gamma).all() and np.array_equal(out[:, :gamma], draft)
+    bad = draft.copy()
+    bad[:, 1] = V + 5
+    acc, out = run_gpu(logits, bad, u, 0.7, 20, 0.8, q=q)
+    assert (acc == 1).all() and (out[:, 1] >= 0).all() and (out[:, 1] < V).all() and (out[:, 2:] == -1).all()
