@@ -593,21 +593,6 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         assert w.status() == 0
         record(f"verify_g{g}:ts_verify_attn", w.bytes, med, mn, w.b.num_seqs * (1 + g),
                {"kv_tokens": w.b.total_tokens, "unit_note": "tokens_per_s counts scored positions B*(1+gamma)"})
-        # the same call 400 times back to back (no flush: 3.2 GB of KV per call): about a quarter of a second
-        # of load, enough for the power cap to pull the SM clock down
-        for _ in range(20):
-            w.attn()
-        torch.cuda.synchronize()
-        with ClockSampler(torch.cuda.current_device(), period_s=0.002) as clk:
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(400):
-                w.attn()
-            b.record()
-            b.synchronize()
-        sus = a.elapsed_time(b) / 400
-        record(f"verify_g{g}:ts_verify_attn_sustained", w.bytes, sus, sus, w.b.num_seqs * (1 + g),
-               {"calls": 400, "clocks": clk.summary()})
         record(f"verify_g{g}:ts_accept_greedy", acc.bytes, amed, amn, emitted,
                {"emitted_tokens": emitted, "accepted_equals_seeded_cuts": bool((acc.acc.cpu().numpy() == acc.cut).all())})
         out[f"verify_g{g}:emitted_tokens_per_s"] = emitted / ((med + amed) * 1e-3)
@@ -690,6 +675,26 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
         out["mixed:split_into_bulk_and_tail_calls"] = {"bulk_ms": mb, "tail_ms": mt, "sum_ms": mb + mt,
                                                        "uniform_ms": out["mixed:ts_decode_attn"]["ms"],
                                                        "tail_seqs": int(len(wt_lens))}
+    # verify attention under sustained load, after everything that is timed call by call (a quarter of a second of
+    # load leaves the SM clock lowered for a while, which the clock-bound selection kernels would pay for)
+    for g in (4, 8, 16):
+        w = W[f"verify_g{g}"]
+        # the same call 400 times back to back (no flush: 3.2 GB of KV per call): about a quarter of a second
+        # of load, enough for the power cap to pull the SM clock down
+        for _ in range(20):
+            w.attn()
+        torch.cuda.synchronize()
+        with ClockSampler(torch.cuda.current_device(), period_s=0.002) as clk:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(400):
+                w.attn()
+            b.record()
+            b.synchronize()
+        sus = a.elapsed_time(b) / 400
+        record(f"verify_g{g}:ts_verify_attn_sustained", w.bytes, sus, sus, w.b.num_seqs * (1 + g),
+               {"calls": 400, "clocks": clk.summary()})
+
     return out
 
 

@@ -468,6 +468,10 @@ static int pick_chunks(long long rows, int vocab)
     if (c > by_len) c = by_len;
     if (c > kMaxChunks) c = kMaxChunks;
     if (c < need) c = need;
+    if (const char *e = getenv("TS_SAMPLE_CHUNKS")) {
+        const long long v = atoll(e);
+        if (v >= need && v <= kMaxChunks) c = v;
+    }
     return (int)c;
 }
 
