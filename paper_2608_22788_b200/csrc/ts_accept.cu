@@ -135,11 +135,12 @@ ts_argmax_reg_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
     const int nvec = end > begin ? (end - begin) >> 3 : 0;
     const uint4 *base = reinterpret_cast<const uint4 *>(logits + (long long)row * row_stride + begin);
     const uint32_t neg_inf2 = 0xff80ff80u;
+    const uint32_t nan2 = 0x7fc07fc0u;       // filler past the chunk's end: NaN never wins and equals nothing
     uint4 v[kVecPerThread];
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
         const int j = threadIdx.x + u * kArgmaxThreads;
-        v[u] = j < nvec ? ld_stream_16B(base + j) : make_uint4(neg_inf2, neg_inf2, neg_inf2, neg_inf2);
+        v[u] = j < nvec ? ld_stream_16B(base + j) : make_uint4(nan2, nan2, nan2, nan2);
     }
     // pass 1: maximum (NaN never wins: max returns the other operand)
     __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162 *>(&neg_inf2);

@@ -59,6 +59,28 @@ def test_odd_vocab_sizes_and_ties(V):
     assert tgt[0, 0] == 0 and tgt[0, 1] == V - 1 and tgt[1, 0] == 0 and tgt[1, 1] == V - 2 and tgt[2, 0] == 0
 
 
+@pytest.mark.parametrize("V", [4096, 20000, 151936])
+def test_nan_never_wins_and_a_row_of_nan_gives_a_token_in_range(V):
+    # NaN logits are outside the contract; what is promised is that they never win against a number, and
+    # that a row without any number still yields index 0 (never an index at or beyond the vocabulary)
+    x = np.full((3, 1, V), np.nan, np.float32)
+    x[1, 0, V - 3] = -np.inf                          # the only number of the row, and the smallest there is
+    x[2, 0, 1::2] = -5.0
+    x[2, 0, 2001] = -4.5
+    bits = wl.f32_to_bf16_bits(x)
+    B = 3
+    lg = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    tgt = torch.full((B, 1), -7, dtype=torch.int32, device="cuda")
+    acc = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    out = torch.full((B, 1), -7, dtype=torch.int32, device="cuda")
+    ws = torch.empty(api.accept_workspace_bytes(B, 0, V), dtype=torch.uint8, device="cuda")
+    api.ts_accept_greedy(lg, None, tgt, acc, out, ws)
+    torch.cuda.synchronize()
+    t = tgt.cpu().numpy()[:, 0]
+    assert t[0] == 0 and t[1] == V - 3 and t[2] == 2001
+    assert np.array_equal(out.cpu().numpy()[:, 0], t) and (acc.cpu().numpy() == 0).all()
+
+
 def test_ties_across_chunk_boundaries_and_signed_zero():
     V = wl.VOCAB
     x = np.full((2, 1, V), -1.0, np.float32)
