@@ -341,12 +341,26 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         best[lane] = 0ull;
         for (int c = lane; c < total; c += 32) cand[c] = src[c];
         __syncwarp();
-        for (int c = lane; c < total; c += 32) {
-            const unsigned long long mine = cand[c];
-            if (mine == 0ull) continue;
-            int rank = 0;
-            for (int j = 0; j < total; ++j) rank += cand[j] > mine;
-            if (rank < top_k) best[rank] = mine;
+        // rank by counting, four candidates per lane against one sweep over the list (a sweep per candidate
+        // made the kernel's longest dependent chain; a binary search per sorted chunk list, with its
+        // dependent probes, measured no faster than that)
+        for (int c0 = 0; c0 < total; c0 += 128) {
+            unsigned long long m[4];
+            int rank[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int c = c0 + 32 * q + lane;
+                m[q] = c < total ? cand[c] : 0ull;
+            }
+#pragma unroll 4
+            for (int j = 0; j < total; ++j) {
+                const unsigned long long x = cand[j];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) rank[q] += x > m[q];
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (m[q] != 0ull && rank[q] < top_k) best[rank[q]] = m[q];
         }
         __syncwarp();
         const unsigned long long key = best[lane];
