@@ -341,26 +341,41 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         best[lane] = 0ull;
         for (int c = lane; c < total; c += 32) cand[c] = src[c];
         __syncwarp();
-        // rank by counting, four candidates per lane against one sweep over the list (a sweep per candidate
-        // made the kernel's longest dependent chain; a binary search per sorted chunk list, with its
-        // dependent probes, measured no faster than that)
-        for (int c0 = 0; c0 < total; c0 += 128) {
-            unsigned long long m[4];
-            int rank[4] = {0, 0, 0, 0};
+        // Merge of the chunks' lists (each sorted in descending order, empty slots = key 0 last).  Only entries
+        // at or above T = the smallest of the lists' m-th entries, m = ceil(top_k / chunks), can be among the
+        // top_k overall (chunks * m >= top_k entries lie at or above T); on random data that is a quarter of
+        // the chunks * top_k candidates.  They are compacted to the front of the list in place and ranked
+        // by counting among themselves (the sweep over all candidates was the longest phase of this kernel:
+        // seventeen warps of one SM issuing it at once).
+        const int mth = (top_k + chunks - 1) / chunks;
+        unsigned long long thr = ~0ull;
+        for (int cc = lane; cc < chunks; cc += 32) {
+            const unsigned long long x = cand[cc * top_k + mth - 1];
+            thr = x < thr ? x : thr;
+        }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int c = c0 + 32 * q + lane;
-                m[q] = c < total ? cand[c] : 0ull;
+        for (int o = 16; o > 0; o >>= 1) { const unsigned long long y = __shfl_xor_sync(FULL, thr, o); thr = y < thr ? y : thr; }
+        int cnt = 0;                                     // a short list (thr == 0) keeps every entry that exists
+        for (int c0 = 0; c0 < total; c0 += 32) {
+            const int c = c0 + lane;
+            const unsigned long long x = c < total ? cand[c] : 0ull;
+            const bool keep = x != 0ull && x >= thr;
+            const unsigned mask = __ballot_sync(FULL, keep);
+            __syncwarp();
+            if (keep) cand[cnt + __popc(mask & ((1u << lane) - 1u))] = x;      // at or before the place it was read from
+            cnt += __popc(mask);
+            __syncwarp();
+        }
+        for (int c = lane; c < cnt; c += 32) {
+            const unsigned long long mine = cand[c];
+            int rank = 0;
+            int j = 0;
+            for (; j + 3 < cnt; j += 4) {
+                const unsigned long long x0 = cand[j], x1 = cand[j + 1], x2 = cand[j + 2], x3 = cand[j + 3];
+                rank += (int)(x0 > mine) + (int)(x1 > mine) + (int)(x2 > mine) + (int)(x3 > mine);
             }
-#pragma unroll 4
-            for (int j = 0; j < total; ++j) {
-                const unsigned long long x = cand[j];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) rank[q] += x > m[q];
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (m[q] != 0ull && rank[q] < top_k) best[rank[q]] = m[q];
+            for (; j < cnt; ++j) rank += cand[j] > mine;
+            if (rank < top_k) best[rank] = mine;
         }
         __syncwarp();
         const unsigned long long key = best[lane];
