@@ -204,6 +204,15 @@ ts_accept_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
                         int B, int gamma, int32_t *target_argmax, int32_t *accept_len, int32_t *out_tokens)
 {
     const int R = gamma + 1;
+    // lane groups of the acceptance step below; a thread's first draft token does not come from the kernel
+    // before, so it is fetched ahead of the wait for it
+    const int lane = threadIdx.x & 31;
+    int g = 1;
+    while (g < R && g < 32) g <<= 1;
+    const int per_warp = 32 / g, sub = lane / g, li = lane % g;
+    const int b_first = (threadIdx.x >> 5) * per_warp + sub;
+    int32_t d_first = -1;
+    if (b_first < B && li < gamma) d_first = draft[(long long)b_first * gamma + li];
     grid_dependency_wait();       // the chunk keys of the kernel before
     for (int r = threadIdx.x; r < B * R; r += blockDim.x) {
         unsigned long long key = 0ull;
@@ -215,10 +224,6 @@ ts_accept_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
     // 32), one lane per position: the draft and target tokens arrive with one round of loads and the first
     // mismatch falls out of a ballot (a thread walking the block position by position paid one memory
     // round trip per accepted token).
-    const int lane = threadIdx.x & 31;
-    int g = 1;
-    while (g < R && g < 32) g <<= 1;
-    const int per_warp = 32 / g, sub = lane / g, li = lane % g;
     const int nslots = (blockDim.x >> 5) * per_warp;
     const unsigned gmask = g == 32 ? 0xffffffffu : ((1u << g) - 1u);
     for (int b0 = (threadIdx.x >> 5) * per_warp; b0 < B; b0 += nslots) {      // warp-uniform trip count
@@ -230,7 +235,8 @@ ts_accept_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         bool found = false;
         for (int i0 = 0; i0 < gamma; i0 += g) {                                // g < 32 only when gamma < g: one pass
             const int i = i0 + li;
-            const bool miss = live && !found && i < gamma && d[i] != t[i];
+            const bool have = i0 == 0 && b == b_first;                          // fetched before the wait
+            const bool miss = live && !found && i < gamma && (have ? d_first : d[i]) != t[i];
             const unsigned m = (__ballot_sync(0xffffffffu, miss) >> (sub * g)) & gmask;
             if (m && !found) { a = i0 + __ffs(m) - 1; found = true; }
         }

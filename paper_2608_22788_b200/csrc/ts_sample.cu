@@ -331,8 +331,21 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
     float *s_q = reinterpret_cast<float *>(smem + (size_t)R * 32 * 8);         // [R][32]: proposal at the kept tokens
     unsigned long long *s_best = reinterpret_cast<unsigned long long *>(smem + (size_t)R * 32 * 12);  // [warps][32]
     unsigned long long *s_cand = s_best + nwarps * 32;                         // [warps][chunks * top_k]
-    grid_dependency_wait();       // the chunk keys of the kernel before
     const int b = blockIdx.x;
+    // warp 0 walks the draft block at the end; the inputs of its first 32 steps do not come from the kernel
+    // before, so they are fetched ahead of the wait for it (lane l holds step l's uniforms, draft token and
+    // that token's proposal probability)
+    float ua_l = 0.f, us_l = 0.f, qx_l = 1.f;
+    int32_t x_l = -1;
+    if (warp == 0 && lane <= gamma) {
+        const float2 u2 = *reinterpret_cast<const float2 *>(uniforms + ((long long)b * R + lane) * 2);
+        ua_l = u2.x;
+        us_l = u2.y;
+        x_l = lane < gamma ? draft[(long long)b * gamma + lane] : -1;
+        if (draft_probs && lane < gamma)
+            qx_l = (x_l >= 0 && x_l < vocab) ? draft_probs[((long long)b * gamma + lane) * q_stride + x_l] : 0.f;
+    }
+    grid_dependency_wait();       // the chunk keys of the kernel before
     for (int i = warp; i < R; i += nwarps) {
         const long long row = (long long)b * R + i;
         const unsigned long long *src = keys + row * total;
@@ -415,11 +428,8 @@ ts_sample_finish_kernel(const unsigned long long *__restrict__ keys, int chunks,
         for (int i = lane; i < R; i += 32) out[i] = -1;
         __syncwarp();
         int a = 0;
-        float ua_l = 0.f, us_l = 0.f;                  // lane l holds the uniforms and the draft of step i0 + l
-        int32_t x_l = -1;
-        float qx_l = 1.f;                              // proposal probability of that draft (1: point proposal)
         for (int i = 0; i <= gamma; ++i) {
-            if ((i & 31) == 0) {
+            if ((i & 31) == 0 && i > 0) {
                 // the next 32 steps' inputs in one round of loads (read inside the walk, each step paid a
                 // memory round trip before it could decide)
                 const int il = i + lane;
