@@ -680,7 +680,10 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
     for g in (4, 8, 16):
         w = W[f"verify_g{g}"]
         # the same call 400 times back to back (no flush: 3.2 GB of KV per call): about a quarter of a second
-        # of load, enough for the power cap to pull the SM clock down
+        # of load, enough for the power cap to pull the SM clock down.  One second of idle first, so that each
+        # depth starts from the same state instead of inheriting the load of the one before
+        torch.cuda.synchronize()
+        time.sleep(1.0)
         for _ in range(20):
             w.attn()
         torch.cuda.synchronize()
