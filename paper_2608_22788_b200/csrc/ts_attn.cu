@@ -668,7 +668,7 @@ __global__ void __launch_bounds__(1024)
 ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__restrict__ gstart,
                      const long long *__restrict__ gpos, const float *__restrict__ part_o,
                      const float *__restrict__ part_lse, uint16_t *out, int B, int q_len, int Hq, int Hkv,
-                     int NG)
+                     int NG, int per_row)
 {
     grid_dependency_wait();       // partials and direct outputs of the attention kernel
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -691,54 +691,83 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     const int k_last = (int)(info & 0xffffu);
     const bool some_empty = (info & 0x40000000u) != 0;
     const int cnt = k_last - k_first + 1;
-    const int nwarps = blockDim.x >> 5;      // one warp per output row of the pair, as many as the pair has rows
-    for (int r = warp; r < rows; r += nwarps) {
-        const int t = r / G, hl = r % G;
-        uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
-        // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
-        // (pair started before them).  Groups whose piece of the tile line is empty (only when W < NG)
-        // wrote nothing: a piece is empty exactly when its start equals the next group's.
-        // Lane i looks at group k_first + i (+ 32, ...): the log-sum-exps come in with one round of loads.
-        float M = -INFINITY;
-        for (int b0 = 0; b0 < cnt; b0 += 32) {
-            const int k = k_first + b0 + lane;
-            float lse = -INFINITY;
-            if (k <= k_last && (!some_empty || gpos[k] != gpos[k + 1]))
-                lse = part_lse[((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r];
-            M = fmaxf(M, lse);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-        constexpr int V = D / 32;
+    // `per_row` warps share an output row of the pair: warp `sub` of them takes the parts sub, sub + per_row, ...
+    // and the partial sums meet in shared memory.  (With one long sequence in the batch a pair is cut into
+    // dozens of parts: one warp walking them in rounds of dependent loads took 35 us for 55 parts.)
+    __shared__ float s_acc[32][D];
+    __shared__ float s_w[32];
+    const int nwarps = blockDim.x >> 5;
+    const int slots = nwarps / per_row;                    // rows in flight at a time
+    const int slot = warp / per_row, sub = warp % per_row;
+    constexpr int V = D / 32;
+    for (int r0 = 0; r0 < rows; r0 += slots) {
+        const int r = r0 + slot;
+        const bool active = r < rows && slot < slots;
         float acc[V];
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] = 0.f;
         float Wsum = 0.f;
-        if (M != -INFINITY) {
+        if (active) {
+            // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
+            // (pair started before them).  Groups whose piece of the tile line is empty (only when W < NG)
+            // wrote nothing: a piece is empty exactly when its start equals the next group's.
+            // Lane i looks at group k_first + i (+ 32, ...): the log-sum-exps come in with one round of loads.
+            float M = -INFINITY;
             for (int b0 = 0; b0 < cnt; b0 += 32) {
-                const int kl = k_first + b0 + lane;
-                float wl = 0.f;
-                if (kl <= k_last && (!some_empty || gpos[kl] != gpos[kl + 1])) {
-                    const float lse = part_lse[((size_t)2 * kl + (kl == k_first ? 1 : 0)) * rows + r];
-                    wl = lse == -INFINITY ? 0.f : expf(lse - M);
-                }
-                const int nj = cnt - b0 < 32 ? cnt - b0 : 32;
-#pragma unroll 4
-                for (int jj = 0; jj < nj; ++jj) {
-                    const float w = __shfl_sync(0xffffffffu, wl, jj);
-                    if (w == 0.f) continue;                       // empty group or empty part: not read
-                    const int k = k_first + b0 + jj;
-                    const float *p = part_o + (((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r) * D + lane * V;
-                    Wsum += w;
+                const int k = k_first + b0 + lane;
+                float lse = -INFINITY;
+                if (k <= k_last && (!some_empty || gpos[k] != gpos[k + 1]))
+                    lse = part_lse[((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r];
+                M = fmaxf(M, lse);
+            }
 #pragma unroll
-                    for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            if (M != -INFINITY) {
+                for (int b0 = 0; b0 < cnt; b0 += 32) {
+                    const int kl = k_first + b0 + lane;
+                    float wl = 0.f;
+                    if (kl <= k_last && (!some_empty || gpos[kl] != gpos[kl + 1])) {
+                        const float lse = part_lse[((size_t)2 * kl + (kl == k_first ? 1 : 0)) * rows + r];
+                        wl = lse == -INFINITY ? 0.f : expf(lse - M);
+                    }
+                    const int nj = cnt - b0 < 32 ? cnt - b0 : 32;
+#pragma unroll 4
+                    for (int jj = sub; jj < nj; jj += per_row) {
+                        const float w = __shfl_sync(0xffffffffu, wl, jj);
+                        if (w == 0.f) continue;                       // empty group or empty part: not read
+                        const int k = k_first + b0 + jj;
+                        const float *p = part_o + (((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r) * D + lane * V;
+                        Wsum += w;
+#pragma unroll
+                        for (int v = 0; v < V; ++v) acc[v] += w * p[v];
+                    }
                 }
             }
         }
-        const float inv = Wsum > 0.f ? 1.f / Wsum : 0.f;
-        uint16_t *o = orow + lane * V;
+        if (per_row > 1) {                                 // CTA-uniform
+            if (active && sub != 0) {
 #pragma unroll
-        for (int v = 0; v < V; v += 2) *reinterpret_cast<uint32_t *>(o + v) = pack_bf16x2(acc[v] * inv, acc[v + 1] * inv);
+                for (int v = 0; v < V; ++v) s_acc[warp][lane * V + v] = acc[v];
+                if (lane == 0) s_w[warp] = Wsum;
+            }
+            __syncthreads();
+            if (active && sub == 0) {
+                for (int o = 1; o < per_row; ++o) {
+                    Wsum += s_w[warp + o];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc[v] += s_acc[warp + o][lane * V + v];
+                }
+            }
+        }
+        if (active && sub == 0) {
+            const int t = r / G, hl = r % G;
+            uint16_t *orow = out + (((size_t)s * q_len + t) * Hq + (size_t)g * G + hl) * D;
+            const float inv = Wsum > 0.f ? 1.f / Wsum : 0.f;
+            uint16_t *o = orow + lane * V;
+#pragma unroll
+            for (int v = 0; v < V; v += 2) *reinterpret_cast<uint32_t *>(o + v) = pack_bf16x2(acc[v] * inv, acc[v + 1] * inv);
+        }
+        if (per_row > 1) __syncthreads();                  // the shared sums are free for the next rows
     }
 }
 
@@ -1173,17 +1202,25 @@ static int run_attention(const ts_attn_params *p, const void *q, const void *k_p
     if (free_mode) {
         const bool overlap = env_int("TS_PDL", 1) != 0;
         const dim3 mgrid((unsigned)NG);
-        const int mwarps = a.rows < 4 ? 4 : (a.rows > 32 ? 32 : a.rows);
+        // one warp per output row of a pair, as many as the pair has rows; when the tile line gives every
+        // (sequence, kv-head) pair many pieces -- few, long sequences -- up to eight warps share a row
+        int mwarps = a.rows < 4 ? 4 : (a.rows > 32 ? 32 : a.rows);
+        const long long pairs = (long long)a.B * a.Hkv;
+        int per_row = 1;
+        if (env_int("TS_MERGE_PER_ROW", 0) > 0) per_row = env_int("TS_MERGE_PER_ROW", 0);
+        else if ((long long)NG >= 4 * pairs) per_row = 8;
+        while (per_row > 1 && (mwarps * per_row > 32 || a.rows > mwarps)) per_row >>= 1;
+        mwarps *= per_row;
         const dim3 mblock((unsigned)mwarps * 32);
         cudaError_t e;
         if (p->head_dim == 128)
             e = launch_overlapped(ts_merge_free_kernel<128>, mgrid, mblock, 0, stream, overlap, a.cum_tiles, a.gstart,
                                   a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
-                                  a.Hkv, NG);
+                                  a.Hkv, NG, per_row);
         else
             e = launch_overlapped(ts_merge_free_kernel<64>, mgrid, mblock, 0, stream, overlap, a.cum_tiles, a.gstart,
                                   a.gpos, (const float *)a.part_o, (const float *)a.part_lse, a.out, a.B, a.q_len, a.Hq,
-                                  a.Hkv, NG);
+                                  a.Hkv, NG, per_row);
         if (e != cudaSuccess) return TS_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
     }
