@@ -651,6 +651,18 @@ def run_extras(torch, api, W, pool, peak, seed, quick=False):
                          "kv_tokens": [r[3] for r in rows], "draws": draws}
     out["concurrency_sweep:ts_decode_attn"] = sweep
 
+    # the end of a rollout step: a handful of long stragglers decode alone (Section 2.1: long tails decode at
+    # low concurrency for a long horizon).  One to four sequences of fixed lengths; the roofline time is the
+    # KV bytes at the measured copy rate, the rest is the three dependent launches (planner, attention, merge)
+    strag = {}
+    for name, ln in (("1x4096", [4096]), ("1x32768", [32768]), ("1x131072", [131072]), ("4x65536", [65536] * 4)):
+        sw = Workload("strag" + name, np.array(ln, np.int32), pool, seed=seed + 300)
+        med, mn = time_with_flush(sw.attn, flush, iters=10, warmup=3)
+        strag[name] = {"ms": med, "ms_min": mn, "tokens_per_s": len(ln) / (med * 1e-3), "GBps": gbs(sw.bytes, med),
+                       "frac_of_measured_peak": gbs(sw.bytes, med) / peak, "roofline_ms": sw.bytes / (peak * 1e6)}
+        del sw
+    out["stragglers:ts_decode_attn"] = strag
+
     # the paper's all-admit completion-time model (Section 2.1, Appendix D) fed with the measured
     # attention-only tau(b): 1024 requests whose remaining lengths follow the mixed pool, 8 replicas,
     # uniform round robin versus top-k tail isolation with 2 of the 8 replicas as the tail pool

@@ -695,7 +695,7 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
     // and the partial sums meet in shared memory.  (With one long sequence in the batch a pair is cut into
     // dozens of parts: one warp walking them in rounds of dependent loads took 35 us for 55 parts.)
     __shared__ float s_acc[32][D];
-    __shared__ float s_w[32];
+    __shared__ float s_w[32], s_m[32];
     const int nwarps = blockDim.x >> 5;
     const int slots = nwarps / per_row;                    // rows in flight at a time
     const int slot = warp / per_row, sub = warp % per_row;
@@ -707,35 +707,38 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] = 0.f;
         float Wsum = 0.f;
+        float M = -INFINITY;                               // largest log-sum-exp among this warp's parts
         if (active) {
             // parts: group k_first wrote slot 2k+1 (pair starts inside it); later groups wrote slot 2k
             // (pair started before them).  Groups whose piece of the tile line is empty (only when W < NG)
             // wrote nothing: a piece is empty exactly when its start equals the next group's.
-            // Lane i looks at group k_first + i (+ 32, ...): the log-sum-exps come in with one round of loads.
-            float M = -INFINITY;
-            for (int b0 = 0; b0 < cnt; b0 += 32) {
-                const int k = k_first + b0 + lane;
+            // This warp's parts are k_first + sub, + per_row, ...; lane i looks at the i-th of them (+ 32, ...),
+            // so that their log-sum-exps come in with one round of loads, and the warp weighs its parts
+            // against its own maximum: the warps of a row are put on a common scale when they meet.
+            const int mine = (cnt - sub + per_row - 1) / per_row;            // parts of this warp
+            for (int b0 = 0; b0 < mine; b0 += 32) {
+                const int k = k_first + sub + (b0 + lane) * per_row;
                 float lse = -INFINITY;
-                if (k <= k_last && (!some_empty || gpos[k] != gpos[k + 1]))
+                if (b0 + lane < mine && (!some_empty || gpos[k] != gpos[k + 1]))
                     lse = part_lse[((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r];
                 M = fmaxf(M, lse);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
             if (M != -INFINITY) {
-                for (int b0 = 0; b0 < cnt; b0 += 32) {
-                    const int kl = k_first + b0 + lane;
+                for (int b0 = 0; b0 < mine; b0 += 32) {
+                    const int kl = k_first + sub + (b0 + lane) * per_row;
                     float wl = 0.f;
-                    if (kl <= k_last && (!some_empty || gpos[kl] != gpos[kl + 1])) {
+                    if (b0 + lane < mine && (!some_empty || gpos[kl] != gpos[kl + 1])) {
                         const float lse = part_lse[((size_t)2 * kl + (kl == k_first ? 1 : 0)) * rows + r];
                         wl = lse == -INFINITY ? 0.f : expf(lse - M);
                     }
-                    const int nj = cnt - b0 < 32 ? cnt - b0 : 32;
+                    const int nj = mine - b0 < 32 ? mine - b0 : 32;
 #pragma unroll 4
-                    for (int jj = sub; jj < nj; jj += per_row) {
+                    for (int jj = 0; jj < nj; ++jj) {
                         const float w = __shfl_sync(0xffffffffu, wl, jj);
                         if (w == 0.f) continue;                       // empty group or empty part: not read
-                        const int k = k_first + b0 + jj;
+                        const int k = k_first + sub + (b0 + jj) * per_row;
                         const float *p = part_o + (((size_t)2 * k + (k == k_first ? 1 : 0)) * rows + r) * D + lane * V;
                         Wsum += w;
 #pragma unroll
@@ -748,14 +751,25 @@ ts_merge_free_kernel(const int32_t *__restrict__ cum_tiles, const GroupStart *__
             if (active && sub != 0) {
 #pragma unroll
                 for (int v = 0; v < V; ++v) s_acc[warp][lane * V + v] = acc[v];
-                if (lane == 0) s_w[warp] = Wsum;
+                if (lane == 0) { s_w[warp] = Wsum; s_m[warp] = M; }
             }
             __syncthreads();
             if (active && sub == 0) {
-                for (int o = 1; o < per_row; ++o) {
-                    Wsum += s_w[warp + o];
+                float Mall = M;
+                for (int o = 1; o < per_row; ++o) Mall = fmaxf(Mall, s_m[warp + o]);
+                if (Mall != -INFINITY) {
+                    const float f0 = M == -INFINITY ? 0.f : expf(M - Mall);
+                    Wsum *= f0;
 #pragma unroll
-                    for (int v = 0; v < V; ++v) acc[v] += s_acc[warp + o][lane * V + v];
+                    for (int v = 0; v < V; ++v) acc[v] *= f0;
+                    for (int o = 1; o < per_row; ++o) {
+                        const float mo = s_m[warp + o];
+                        if (mo == -INFINITY) continue;
+                        const float f = expf(mo - Mall);
+                        Wsum += f * s_w[warp + o];
+#pragma unroll
+                        for (int v = 0; v < V; ++v) acc[v] += f * s_acc[warp + o][lane * V + v];
+                    }
                 }
             }
         }
