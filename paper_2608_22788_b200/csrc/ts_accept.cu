@@ -120,8 +120,11 @@ ts_argmax_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride
 // use -- finds the chunk maximum with packed bf16x2 max instructions, then the first position equal
 // to it with packed compares.  About 13 instructions per 16 bytes instead of ~80 for the generic
 // key-per-element scan, which keeps the kernel bandwidth-bound.
-constexpr int kVecPerThread = 16;
-constexpr int kFastChunk = kArgmaxThreads * kVecPerThread * 8;      // elements per chunk (32768)
+// Eight vectors per thread: 52 registers, four CTAs per SM.  Sixteen (a 32768-element chunk, 79 registers,
+// three CTAs per SM) measured 2 us slower per call at 144 and 272 rows, four to twelve the same as eight
+// or slower: with more, shorter-lived CTAs on an SM their load and reduce phases interleave better.
+constexpr int kVecPerThread = 8;
+constexpr int kFastChunk = kArgmaxThreads * kVecPerThread * 8;      // elements per chunk (16384)
 
 __global__ void __launch_bounds__(kArgmaxThreads)
 ts_argmax_reg_kernel(const uint16_t *__restrict__ logits, long long row_stride, int vocab, int chunk_len,
