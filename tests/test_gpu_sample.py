@@ -318,3 +318,28 @@ def test_proposal_equal_to_target_accepts_everything_and_out_of_range_draft_is_r
     bad[:, 1] = V + 5
     acc, out = run_gpu(logits, bad, u, 0.7, 20, 0.8, q=q)
     assert (acc == 1).all() and (out[:, 1] >= 0).all() and (out[:, 1] < V).all() and (out[:, 2:] == -1).all()
+
+
+@pytest.mark.parametrize("with_q", [False, True])
+def test_long_draft_blocks_reload_the_walk_inputs(with_q):
+    # gamma above 32: the walk fetches its inputs 32 steps at a time; drafts that mostly agree with the target so
+    # that the walk gets past the first batch of steps
+    B, gamma, V = 12, 45, 4096
+    rng = np.random.default_rng(77)
+    logits = wl.make_logits(B, gamma, V, seed=77)
+    f = wl.bf16_bits_to_f32(logits)
+    best = np.argmax(f, -1)
+    # sharpen: make the row maximum dominate so that it is accepted with probability near one
+    x = f.copy()
+    np.put_along_axis(x, best[..., None], 30.0, axis=-1)
+    logits = wl.f32_to_bf16_bits(x)
+    draft = best[:, :gamma].astype(np.int32).copy()
+    draft[3, 40] = (draft[3, 40] + 1) % V                  # one late rejection
+    draft[5, 33] = (draft[5, 33] + 7) % V
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    q = None
+    if with_q:
+        q = np.full((B, gamma, V), 0.2 / (V - 1), np.float32)
+        np.put_along_axis(q, draft[..., None].astype(np.int64), 0.8, axis=-1)
+    acc, out = check(logits, draft, u, 0.7, 20, 0.8, q=q)
+    assert acc.max() == gamma and acc[3] == 40 and acc[5] == 33
