@@ -244,3 +244,20 @@ def test_both_verify_kernels_agree_with_the_oracle(monkeypatch):
     assert_close(DeviceBatch(b).verify(), ref, "tcgen05")
     monkeypatch.setenv("TS_ATTN_TC", "0")
     assert_close(DeviceBatch(b).verify(), ref, "warp mma")
+
+
+# ------------------------------------------------------------------ one long straggler
+@pytest.mark.parametrize("per_row", [0, 1, 2, 8])
+@pytest.mark.parametrize("ql", [1, 4])
+def test_one_long_sequence_is_cut_into_dozens_of_parts(per_row, ql, monkeypatch):
+    # The end of a rollout step: one sequence, every (sequence, kv-head) pair spread over dozens of warp
+    # groups.  The merge then has more parts per row than lanes in a round of loads when a single warp
+    # walks them (per_row = 1), and shares them among several warps otherwise (0 = the library's choice).
+    if per_row:
+        monkeypatch.setenv("TS_MERGE_PER_ROW", str(per_row))
+    b = wl.make_batch("lone", [70001 + ql], q_len=ql, num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=64,
+                      seed=90 + ql, poison=True)
+    ref, _ = oracle.attention_batch(b)
+    d = DeviceBatch(b)
+    out = d.verify() if ql > 1 else d.decode()
+    assert_close(out, ref, f"one long sequence, per_row={per_row}, q_len={ql}")
