@@ -92,18 +92,18 @@ __device__ __noinline__ void push_candidates(uint4 v, uint32_t e0, uint32_t e1, 
                                              int *cnt, unsigned long long *cand, uint32_t present, const uint16_t *rowp,
                                              float pen)
 {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    const uint32_t e[4] = {e0, e1, e2, e3};
-    for (int i = 0; i < 4; ++i) {
-        if (e[i] & 0xffffu) {
-            const int s = atomicAdd(cnt, 1);
-            if (s < kCap) cand[s] = pack_key(element_key(w[i], (present >> (2 * i)) & 1u, rowp, idx0 + 2 * i, pen), idx0 + 2 * i);
-        }
-        if (e[i] >> 16) {
-            const int s = atomicAdd(cnt, 1);
-            if (s < kCap)
-                cand[s] = pack_key(element_key(w[i] >> 16, (present >> (2 * i + 1)) & 1u, rowp, idx0 + 2 * i + 1, pen), idx0 + 2 * i + 1);
-        }
+    // one bit per element that passed the threshold test (almost always a single one): the loop runs once per
+    // candidate instead of visiting all eight slots
+    uint32_t b8 = (e0 & 1u) | ((e0 >> 15) & 2u) | ((e1 & 1u) << 2) | ((e1 >> 13) & 8u) |
+                  ((e2 & 1u) << 4) | ((e2 >> 11) & 0x20u) | ((e3 & 1u) << 6) | ((e3 >> 9) & 0x80u);
+    while (b8) {
+        const int i = __ffs(b8) - 1;
+        b8 &= b8 - 1u;
+        const int wi = i >> 1;
+        const uint32_t word = wi == 0 ? v.x : (wi == 1 ? v.y : (wi == 2 ? v.z : v.w));
+        const uint32_t bits = (i & 1) ? word >> 16 : word;
+        const int s = atomicAdd(cnt, 1);
+        if (s < kCap) cand[s] = pack_key(element_key(bits, (present >> i) & 1u, rowp, idx0 + i, pen), idx0 + i);
     }
 }
 
