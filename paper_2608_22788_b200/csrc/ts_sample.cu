@@ -88,7 +88,7 @@ __device__ __forceinline__ unsigned long long pack_key(uint32_t key16, int idx)
     return ((unsigned long long)key16 << 32) | (unsigned long long)(0xffffffffu - (uint32_t)idx);
 }
 
-__device__ __noinline__ void push_candidates(uint4 v, uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, int idx0,
+__device__ __forceinline__ void push_candidates(uint4 v, uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, int idx0,
                                              int *cnt, unsigned long long *cand, uint32_t present, const uint16_t *rowp,
                                              float pen)
 {
@@ -245,7 +245,7 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
     // ---- threshold T1 = the top_k-th largest of the 256 thread maxima (0 if fewer than top_k threads
     //      hold a number): the top_k-th largest element of the chunk is >= T1, so the chunk's top_k are
     //      all >= T1, and on random data only a few dozen elements are.  Warp 0 finds it by binary search
-    //      on the 17-bit key, counting with ballots over the 8 maxima each of its lanes holds.
+    //      on the 17-bit key, each lane counting over the 8 maxima it holds.
     s_tkey[tid] = tkey;
     __syncthreads();
     if (tid < 32) {
@@ -263,7 +263,8 @@ ts_topk_chunk_kernel(const uint16_t *__restrict__ logits, long long row_stride, 
             const uint32_t mid = (lo + hi) >> 1;
             int c = 0;
 #pragma unroll
-            for (int i = 0; i < kThreads / 32; ++i) c += __popc(__ballot_sync(0xffffffffu, k8[i] >= mid));
+            for (int i = 0; i < kThreads / 32; ++i) c += k8[i] >= mid;
+            c = __reduce_add_sync(0xffffffffu, c);           // one warp-wide add instead of a ballot per key
             if (c >= want) lo = mid; else hi = mid;
         }
         if (tid == 0) s_t1 = lo;
