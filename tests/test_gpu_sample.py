@@ -343,3 +343,19 @@ def test_long_draft_blocks_reload_the_walk_inputs(with_q):
         np.put_along_axis(q, draft[..., None].astype(np.int64), 0.8, axis=-1)
     acc, out = check(logits, draft, u, 0.7, 20, 0.8, q=q)
     assert acc.max() == gamma and acc[3] == 40 and acc[5] == 33
+
+
+@pytest.mark.parametrize("pen", [1.2, 0.3, 1.5, -0.7])
+def test_presence_penalties_that_are_and_are_not_bf16_numbers(pen):
+    # 1.5 is a bf16 number, 1.2, 0.3 and -0.7 are not: the lowered logits are then no bf16 numbers either and
+    # only the exact fp32 keys order them; the row maxima are among the seen tokens, so the penalty decides
+    B, gamma, V = 16, 4, 32768
+    rng = np.random.default_rng(int(abs(pen) * 100))
+    logits = wl.make_logits(B, gamma, V, seed=21)
+    best = np.argmax(wl.bf16_bits_to_f32(logits), -1)
+    draft = np.where(rng.random((B, gamma)) < 0.7, best[:, :gamma], rng.integers(0, V, (B, gamma))).astype(np.int32)
+    bits = rng.random((B, V)) < 0.05
+    bits[np.arange(B)[:, None], best] = True               # the row maxima are among the seen tokens
+    seen = np.packbits(bits, axis=1, bitorder="little")
+    u = rng.random((B, gamma + 1, 2), dtype=np.float32)
+    check(logits, draft, u, 0.7, 20, 0.8, seen=seen, pen=pen)
